@@ -1,0 +1,144 @@
+// Activation prologue (Section 4.4, first kernel; Eq. 8; Eq. 1): one pass over X that applies the
+// inverse channel scaling D^-1 and the stream gain gamma_{tau,s(i)}, finds the row range, and writes
+// only the integer codes Q_X and the row scale r_i = Delta_X / gamma_{s(i)}.
+//
+// HBM-bound: one warp owns one row; every lane moves 16 bytes (8 bf16) per step so that a warp reads
+// 512 contiguous bytes and writes 256 contiguous bytes of codes.  The raw row stays in registers
+// between the range pass and the rounding pass (rows up to 8192 channels; longer rows are read a
+// second time, from L2).  All fp32 operations are individually rounded, in the order
+// v = (x * dinv) * gamma, q = rint(v * (q_max / a)), r = (a / q_max) / gamma.
+#include "internal.cuh"
+
+namespace rudder {
+
+__device__ __forceinline__ uint4 ld_nc_16(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ int stream_of_row(const SegParams& seg, int row) {
+    int s = 0;
+    for (int i = 1; i < seg.n_seg; ++i)
+        if (row >= seg.offset[i]) s = i;
+    return seg.stream[s];
+}
+
+// 8 bf16 (one uint4) x 8 channel scales x gain -> 8 fp32
+__device__ __forceinline__ void scale8(const uint4& x, const float4& d0, const float4& d1, float g, float (&v)[8]) {
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+    const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16);
+        const float hi = __uint_as_float(w[i] & 0xFFFF0000u);
+        v[2 * i] = __fmul_rn(__fmul_rn(lo, dd[2 * i]), g);
+        v[2 * i + 1] = __fmul_rn(__fmul_rn(hi, dd[2 * i + 1]), g);
+    }
+}
+
+__device__ __forceinline__ uint2 round8(const float (&v)[8], float inv, int qmax) {
+    uint32_t out[2] = {0u, 0u};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        int q = __float2int_rn(__fmul_rn(v[i], inv));
+        q = max(-qmax, min(qmax, q));
+        out[i >> 2] |= (static_cast<uint32_t>(q) & 0xFFu) << (8 * (i & 3));
+    }
+    return make_uint2(out[0], out[1]);
+}
+
+// NIT = number of 256-channel steps whose raw data is kept in registers (0: re-read the row).
+template <int NIT>
+__global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int8_t* __restrict__ codes, int64_t ldc,
+                                                        float* __restrict__ r)
+{
+    const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= a.M) return;
+    const float g = a.gamma_step[stream_of_row(a.seg, row)];
+    const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(row) * a.ldx);
+    const float4* dv = reinterpret_cast<const float4*>(a.dinv);
+    const int n_chunks = a.K >> 3;                 // 16-byte chunks in the row
+    const int n_it = (n_chunks + 31) >> 5;
+
+    uint4 xr[NIT > 0 ? NIT : 1];
+    float amax = 0.0f;
+    if (a.clip_step == nullptr || NIT > 0) {
+        if (NIT > 0) {
+#pragma unroll
+            for (int it = 0; it < NIT; ++it) {
+                const int c = it * 32 + lane;
+                if (c < n_chunks) xr[it] = ld_nc_16(xrow + c);
+            }
+        }
+        if (a.clip_step == nullptr) {
+            if (NIT > 0) {
+#pragma unroll
+                for (int it = 0; it < NIT; ++it) {
+                    const int c = it * 32 + lane;
+                    if (c < n_chunks) {
+                        float v[8];
+                        scale8(xr[it], __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+                    }
+                }
+            } else {
+                for (int it = 0; it < n_it; ++it) {
+                    const int c = it * 32 + lane;
+                    if (c < n_chunks) {
+                        float v[8];
+                        scale8(ld_nc_16(xrow + c), __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
+                    }
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        }
+    }
+    const float range = a.clip_step ? *a.clip_step : amax;     // a_i: shared threshold c_tau, or the row's absmax
+    const float inv = (range != 0.0f) ? __fdiv_rn(static_cast<float>(qmax), range) : 0.0f;
+    uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldc);
+
+    if (NIT > 0) {
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int c = it * 32 + lane;
+            if (c < n_chunks) {
+                float v[8];
+                scale8(xr[it], __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
+                crow[c] = round8(v, inv, qmax);
+            }
+        }
+    } else {
+        for (int it = 0; it < n_it; ++it) {
+            const int c = it * 32 + lane;
+            if (c < n_chunks) {
+                float v[8];
+                scale8(ld_nc_16(xrow + c), __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
+                crow[c] = round8(v, inv, qmax);
+            }
+        }
+    }
+    if (lane == 0)
+        r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, static_cast<float>(qmax)), g) : 0.0f;
+}
+
+cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st)
+{
+    const int threads = 256;
+    const int blocks = (a.M * 32 + threads - 1) / threads;
+    const int n_it = (a.K / 8 + 31) / 32;
+    if (n_it <= 4)       actq_int_kernel<4><<<blocks, threads, 0, st>>>(a, qmax, codes, ldc, r);
+    else if (n_it <= 8)  actq_int_kernel<8><<<blocks, threads, 0, st>>>(a, qmax, codes, ldc, r);
+    else if (n_it <= 16) actq_int_kernel<16><<<blocks, threads, 0, st>>>(a, qmax, codes, ldc, r);
+    else if (n_it <= 32) actq_int_kernel<32><<<blocks, threads, 0, st>>>(a, qmax, codes, ldc, r);
+    else                 actq_int_kernel<0><<<blocks, threads, 0, st>>>(a, qmax, codes, ldc, r);
+    return cudaGetLastError();
+}
+
+}  // namespace rudder

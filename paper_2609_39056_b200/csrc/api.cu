@@ -1,0 +1,350 @@
+// Host side of the C ABI: argument checks, tensor maps, workspace carving, launches.
+#include "internal.cuh"
+
+#include <stdlib.h>
+#include <string.h>
+
+using namespace rudder;
+
+namespace {
+
+// ---- cuTensorMapEncodeTiled through the runtime (no link-time dependency on the driver library) --
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Row-major 2D tensor [rows, cols] of `esize`-byte elements; box = {box_cols, box_rows}.
+bool make_tmap_2d(CUtensorMap* tm, CUtensorMapDataType dt, int esize, const void* base, uint64_t cols, uint64_t rows,
+                  uint64_t row_stride_bytes, uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle sw)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    (void)esize;
+    cuuint64_t gdim[2] = {cols, rows};
+    cuuint64_t gstride[1] = {row_stride_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, dt, 2, const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool g_gemm_ready[64] = {false};
+
+rudder_status ensure_init()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return RUDDER_ERR_CUDA;
+    if (!g_gemm_ready[dev]) {
+        if (gemm_i8_init() != cudaSuccess) return RUDDER_ERR_CUDA;
+        g_gemm_ready[dev] = true;
+    }
+    return RUDDER_OK;
+}
+
+rudder_status check_table_and_segments(const rudder_segments* seg, int step, const rudder_scale_table* tab, int M,
+                                       SegParams* out)
+{
+    if (!seg || !tab || !tab->gamma || !seg->seg_offsets || !seg->seg_stream) return RUDDER_ERR_ARG;
+    if (tab->T < 1 || tab->S < 1 || tab->S > kMaxStreams) return RUDDER_ERR_ARG;
+    if (step < 0 || step >= tab->T) return RUDDER_ERR_ARG;
+    if (tab->mode != RUDDER_RANGE_PER_TOKEN && tab->mode != RUDDER_RANGE_STATIC) return RUDDER_ERR_ARG;
+    if (tab->mode == RUDDER_RANGE_STATIC && !tab->clip) return RUDDER_ERR_ARG;
+    if (seg->n_seg < 1 || seg->n_seg > kMaxSeg) return RUDDER_ERR_ARG;
+    if (seg->seg_offsets[0] != 0 || seg->seg_offsets[seg->n_seg] != M) return RUDDER_ERR_ARG;
+    out->n_seg = seg->n_seg;
+    for (int i = 0; i < seg->n_seg; ++i) {
+        if (seg->seg_offsets[i + 1] < seg->seg_offsets[i]) return RUDDER_ERR_ARG;
+        if (seg->seg_stream[i] < 0 || seg->seg_stream[i] >= tab->S) return RUDDER_ERR_ARG;
+        out->offset[i] = seg->seg_offsets[i];
+        out->stream[i] = seg->seg_stream[i];
+    }
+    out->offset[seg->n_seg] = M;
+    for (int i = seg->n_seg + 1; i <= kMaxSeg; ++i) out->offset[i] = M;
+    for (int i = seg->n_seg; i < kMaxSeg; ++i) out->stream[i] = 0;
+    return RUDDER_OK;
+}
+
+int qmax_of(int scheme) { return scheme == RUDDER_W4A8_INT ? 127 : 7; }
+
+struct LinearPlan {
+    SegParams seg;
+    size_t off_codes, off_r, bytes;
+};
+
+size_t workspace_bytes_for(const rudder_weight* w, int M)
+{
+    if (!w || M < 1) return 0;
+    const size_t codes = align_up(static_cast<size_t>(M) * w->K, 256);
+    const size_t r = align_up(static_cast<size_t>(M) * sizeof(float), 256);
+    return codes + r;
+}
+
+rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M, const rudder_segments* seg,
+                          int step, const rudder_scale_table* tab, const float* bias, uint16_t* Y, int64_t ldy,
+                          void* workspace, size_t workspace_bytes, cudaStream_t st, int32_t* acc, int row0, int rows,
+                          int col0, int cols)
+{
+    if (!w || !X || !Y) return RUDDER_ERR_ARG;
+    if (M < 1) return RUDDER_ERR_SHAPE;
+    SegParams sp;
+    rudder_status s = check_table_and_segments(seg, step, tab, M, &sp);
+    if (s != RUDDER_OK) return s;
+    if (!aligned(X, 16) || !aligned(Y, 16) || ldx % 8 != 0 || ldy % 8 != 0 || ldx < w->K || ldy < w->N) return RUDDER_ERR_ALIGN;
+    if (bias && !aligned(bias, 16)) return RUDDER_ERR_ALIGN;
+    if (w->scheme != RUDDER_W4A8_INT && w->scheme != RUDDER_W4A4_INT) return RUDDER_ERR_UNSUPPORTED;
+    const size_t need = workspace_bytes_for(w, M);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return RUDDER_ERR_WORKSPACE;
+    if (acc) {
+        if (rows < 1 || cols < 1 || row0 < 0 || col0 < 0 || row0 % 128 != 0 || col0 % 64 != 0) return RUDDER_ERR_ARG;
+    }
+    s = ensure_init();
+    if (s != RUDDER_OK) return s;
+
+    int8_t* codes = static_cast<int8_t*>(workspace);
+    float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
+
+    ActqArgs a;
+    a.X = X; a.ldx = ldx; a.M = M; a.K = w->K; a.dinv = w->dinv;
+    a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
+    a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;
+    a.seg = sp;
+    if (launch_actq_int(a, qmax_of(w->scheme), codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+
+    GemmI8Args g;
+    if (!make_tmap_2d(&g.tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(M),
+                      static_cast<uint64_t>(w->K), 128, static_cast<uint32_t>(M < 128 ? M : 128), CU_TENSOR_MAP_SWIZZLE_128B))
+        return RUDDER_ERR_CUDA;
+    g.wt = w->tiles;
+    g.M = M; g.N = w->N; g.K = w->K; g.G = w->G;
+    g.row_scale = r; g.bias = bias; g.Y = Y; g.ldy = ldy;
+    g.acc = acc; g.row0 = row0; g.rows = rows; g.col0 = col0; g.cols = cols;
+    if (launch_gemm_i8(g, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    return RUDDER_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rudder_status_string(rudder_status s)
+{
+    switch (s) {
+        case RUDDER_OK: return "ok";
+        case RUDDER_ERR_ARG: return "invalid argument";
+        case RUDDER_ERR_SHAPE: return "unsupported shape";
+        case RUDDER_ERR_ALIGN: return "misaligned pointer or leading dimension";
+        case RUDDER_ERR_UNSUPPORTED: return "unsupported scheme or mode";
+        case RUDDER_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case RUDDER_ERR_CUDA: return "CUDA call failed";
+        case RUDDER_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    }
+    return "unknown status";
+}
+
+rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, rudder_scheme scheme, int group,
+                                  void* stream, rudder_weight** out)
+{
+    if (out) *out = nullptr;
+    if (!W || !out) return RUDDER_ERR_ARG;
+    if (N < 64 || N % 64 != 0 || K < 128 || K % 128 != 0) return RUDDER_ERR_SHAPE;
+    if (scheme != RUDDER_W4A8_INT && scheme != RUDDER_W4A4_INT) return RUDDER_ERR_UNSUPPORTED;
+    if (!(group == 64 || group == 128 || group == K)) return RUDDER_ERR_SHAPE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rudder_status s = ensure_init();
+    if (s != RUDDER_OK) return s;
+
+    rudder_weight* w = static_cast<rudder_weight*>(calloc(1, sizeof(rudder_weight)));
+    if (!w) return RUDDER_ERR_CUDA;
+    w->N = N; w->K = K; w->G = group; w->scheme = scheme;
+    cudaGetDevice(&w->device);
+    const size_t n_groups = static_cast<size_t>(K / group);
+    const size_t code_bytes = static_cast<size_t>(N) * (K / 2);
+    int8_t* tmp = nullptr;
+    bool ok = cudaMalloc(&w->codes, code_bytes) == cudaSuccess &&
+              cudaMalloc(&w->scales_t, n_groups * N * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&w->scales_c, n_groups * N * sizeof(uint16_t)) == cudaSuccess &&
+              cudaMalloc(&w->dinv, static_cast<size_t>(K) * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&w->tensor_scale, sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&tmp, static_cast<size_t>(N) * K) == cudaSuccess;
+    w->bytes = code_bytes + n_groups * N * (sizeof(float) + sizeof(uint16_t)) + static_cast<size_t>(K) * sizeof(float) + sizeof(float);
+    if (ok) {
+        const float one = 1.0f;
+        ok = cudaMemcpyAsync(w->tensor_scale, &one, sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess &&
+             launch_pack_int4(W, d, N, K, group, w->codes, w->scales_t, static_cast<uint16_t*>(w->scales_c), w->dinv, tmp, st) == cudaSuccess &&
+             cudaStreamSynchronize(st) == cudaSuccess;
+    }
+    if (tmp) cudaFree(tmp);
+    if (ok) {
+        for (int t = 0; t < 2 && ok; ++t) {
+            const int nt = t == 0 ? 128 : 256;
+            w->tiles[t].n_tile = nt;
+            const uint32_t box_rows = static_cast<uint32_t>(N < nt ? N : nt);
+            ok = make_tmap_2d(&w->tiles[t].codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w->codes, static_cast<uint64_t>(K / 2),
+                              static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), 64, box_rows, CU_TENSOR_MAP_SWIZZLE_NONE) &&
+                 make_tmap_2d(&w->tiles[t].scales, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w->scales_t, static_cast<uint64_t>(N),
+                              static_cast<uint64_t>(n_groups), static_cast<uint64_t>(N) * sizeof(float), box_rows, 1,
+                              CU_TENSOR_MAP_SWIZZLE_NONE);
+        }
+    }
+    if (!ok) {
+        rudder_weight_free(w);
+        return RUDDER_ERR_CUDA;
+    }
+    *out = w;
+    return RUDDER_OK;
+}
+
+rudder_status rudder_weight_free(rudder_weight* w)
+{
+    if (!w) return RUDDER_OK;
+    cudaFree(w->codes);
+    cudaFree(w->scales_t);
+    cudaFree(w->scales_c);
+    cudaFree(w->sf_tiled);
+    cudaFree(w->dinv);
+    cudaFree(w->tensor_scale);
+    free(w);
+    return RUDDER_OK;
+}
+
+rudder_status rudder_weight_info(const rudder_weight* w, int* N, int* K, int* group, int* scheme, size_t* device_bytes)
+{
+    if (!w) return RUDDER_ERR_ARG;
+    if (N) *N = w->N;
+    if (K) *K = w->K;
+    if (group) *group = w->G;
+    if (scheme) *scheme = w->scheme;
+    if (device_bytes) *device_bytes = w->bytes;
+    return RUDDER_OK;
+}
+
+rudder_status rudder_weight_export(const rudder_weight* w, uint8_t* codes, void* scales, float* dinv, float* tensor_scale,
+                                   void* stream)
+{
+    if (!w) return RUDDER_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (codes && launch_export_int4(w->codes, w->N, w->K, codes, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    const size_t n_groups = static_cast<size_t>(w->K / w->G);
+    if (scales && cudaMemcpyAsync(scales, w->scales_c, n_groups * w->N * sizeof(uint16_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
+    if (dinv && cudaMemcpyAsync(dinv, w->dinv, static_cast<size_t>(w->K) * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
+    if (tensor_scale && cudaMemcpyAsync(tensor_scale, w->tensor_scale, sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
+    return RUDDER_OK;
+}
+
+size_t rudder_linear_workspace_bytes(const rudder_weight* w, int M) { return workspace_bytes_for(w, M); }
+
+rudder_status rudder_linear(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M, const rudder_segments* seg,
+                            int step, const rudder_scale_table* tab, const float* bias, uint16_t* Y, int64_t ldy,
+                            void* workspace, size_t workspace_bytes, void* stream)
+{
+    return linear_impl(w, X, ldx, M, seg, step, tab, bias, Y, ldy, workspace, workspace_bytes,
+                       static_cast<cudaStream_t>(stream), nullptr, 0, 0, 0, 0);
+}
+
+rudder_status rudder_linear_dump_acc(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M,
+                                     const rudder_segments* seg, int step, const rudder_scale_table* tab,
+                                     const float* bias, uint16_t* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                     void* stream, int row0, int rows, int col0, int cols, int32_t* acc)
+{
+    if (!acc) return RUDDER_ERR_ARG;
+    return linear_impl(w, X, ldx, M, seg, step, tab, bias, Y, ldy, workspace, workspace_bytes,
+                       static_cast<cudaStream_t>(stream), acc, row0, rows, col0, cols);
+}
+
+size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M)
+{
+    if (!args || M < 1) return 0;
+    size_t total = 0;
+    for (int l = 0; l < 4; ++l) {
+        if (!args->w[l]) return 0;
+        total += workspace_bytes_for(args->w[l], M);
+    }
+    return total;
+}
+
+rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_segments* seg, int step, void* workspace,
+                           size_t workspace_bytes, void* stream)
+{
+    if (!args) return RUDDER_ERR_ARG;
+    for (int l = 0; l < 4; ++l)
+        if (!args->w[l] || !args->tab[l] || !args->x[l] || !args->y[l]) return RUDDER_ERR_ARG;
+    const size_t need = rudder_block_workspace_bytes(args, M);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need || need == 0) return RUDDER_ERR_WORKSPACE;
+    // validate everything before the first launch
+    for (int l = 0; l < 4; ++l) {
+        SegParams sp;
+        rudder_status s = check_table_and_segments(seg, step, args->tab[l], M, &sp);
+        if (s != RUDDER_OK) return s;
+        const rudder_weight* w = args->w[l];
+        if (!aligned(args->x[l], 16) || !aligned(args->y[l], 16) || args->ldx[l] % 8 != 0 || args->ldy[l] % 8 != 0 ||
+            args->ldx[l] < w->K || args->ldy[l] < w->N)
+            return RUDDER_ERR_ALIGN;
+    }
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    for (int l = 0; l < 4; ++l) {
+        const size_t bytes = workspace_bytes_for(args->w[l], M);
+        rudder_status s = rudder_linear(args->w[l], args->x[l], args->ldx[l], M, seg, step, args->tab[l], args->bias[l],
+                                        args->y[l], args->ldy[l], ws, bytes, stream);
+        if (s != RUDDER_OK) return s;
+        ws += bytes;
+    }
+    return RUDDER_OK;
+}
+
+rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M,
+                                          const rudder_segments* seg, int step, const rudder_scale_table* tab,
+                                          void* codes, uint8_t* block_scales, float* row_scale, void* stream)
+{
+    (void)block_scales;
+    if (!w || !X || !codes || !row_scale) return RUDDER_ERR_ARG;
+    if (M < 1) return RUDDER_ERR_SHAPE;
+    SegParams sp;
+    rudder_status s = check_table_and_segments(seg, step, tab, M, &sp);
+    if (s != RUDDER_OK) return s;
+    if (!aligned(X, 16) || ldx % 8 != 0 || ldx < w->K || !aligned(codes, 16)) return RUDDER_ERR_ALIGN;
+    if (w->scheme != RUDDER_W4A8_INT && w->scheme != RUDDER_W4A4_INT) return RUDDER_ERR_UNSUPPORTED;
+    ActqArgs a;
+    a.X = X; a.ldx = ldx; a.M = M; a.K = w->K; a.dinv = w->dinv;
+    a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
+    a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;
+    a.seg = sp;
+    if (launch_actq_int(a, qmax_of(w->scheme), static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
+    return RUDDER_OK;
+}
+
+rudder_status rudder_device_status(int* last, int* where)
+{
+    if (!last) return RUDDER_ERR_ARG;
+    int v[2] = {0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) return RUDDER_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(v, rudder::g_device_status, sizeof(v)) != cudaSuccess) return RUDDER_ERR_CUDA;
+    const int zero[2] = {0, 0};
+    if (cudaMemcpyToSymbol(rudder::g_device_status, zero, sizeof(zero)) != cudaSuccess) return RUDDER_ERR_CUDA;
+    *last = v[0];
+    if (where) *where = v[1];
+    return RUDDER_OK;
+}
+
+}  // extern "C"

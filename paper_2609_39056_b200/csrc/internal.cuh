@@ -1,0 +1,89 @@
+// Host-side declarations shared by the translation units of the library (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/rudder.h"
+
+namespace rudder {
+
+constexpr int kMaxSeg = 64;
+constexpr int kMaxStreams = 16;
+
+// Row -> stream map, passed by value in kernel parameters (no device allocation, graph-capturable).
+struct SegParams {
+    int n_seg;
+    int offset[kMaxSeg + 1];
+    int stream[kMaxSeg];
+};
+
+// What a packed weight holds on the device.  Layouts are private to the kernels:
+//   codes     integer schemes: [N, K/2] bytes; inside every run of 32 input channels, byte b (0..15)
+//             holds channel b in its low nibble and channel 16 + b in its high nibble (two's
+//             complement), so that one 16-byte load expands into two 16-byte rows of int8 with two
+//             logic operations per word.  NVFP4: [N, K/2] bytes, low nibble = even channel (E2M1).
+//   scales_t  integer schemes: fp32 [K/G, N] = Delta_W[j,g] / 16 (the kernel feeds the tensor core
+//             16 x the code: the nibble placed in the top half of the byte).
+//   scales_c  integer schemes: fp16 [N, K/G] canonical copy.  NVFP4: UE4M3 [N, K/16] canonical copy.
+//   sf_tiled  NVFP4: UE4M3 scale factors in the tensor core's tiled order:
+//             [N/128][K/64][32 lanes][4 row-quarters][4 blocks] bytes.
+//   dinv      fp32 [K]
+struct WeightTiles {
+    CUtensorMap codes;    // packed codes, box = {64 bytes, n_tile rows}
+    CUtensorMap scales;   // scales_t, box = {n_tile floats, 1 group}
+    int n_tile;
+};
+}  // namespace rudder
+
+struct rudder_weight {
+    int N, K, G, scheme;
+    int device;
+    uint8_t* codes;
+    float* scales_t;
+    void* scales_c;
+    uint8_t* sf_tiled;
+    float* dinv;
+    float* tensor_scale;      // device [1]
+    size_t bytes;
+    rudder::WeightTiles tiles[2];   // [0]: n_tile = 128, [1]: n_tile = 256
+};
+
+namespace rudder {
+
+struct ActqArgs {
+    const uint16_t* X;
+    int64_t ldx;
+    int M, K;
+    const float* dinv;
+    const float* gamma_step;   // gamma + step * S
+    const float* clip_step;    // clip + step, or nullptr (per-token range)
+    SegParams seg;
+};
+
+// ---- launches (each returns cudaGetLastError of its launch) ----------------------------------
+cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G, uint8_t* codes_il,
+                             float* scales_t, uint16_t* scales_c, float* dinv, int8_t* tmp_codes,
+                             cudaStream_t st);
+cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, cudaStream_t st);
+
+cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);
+
+struct GemmI8Args {
+    CUtensorMap tm_a;           // activation codes int8 [M, K], box {128, 128}, 128-byte swizzle
+    const WeightTiles* wt;
+    int M, N, K, G;
+    const float* row_scale;     // r [M]
+    const float* bias;          // [N] or nullptr
+    uint16_t* Y;
+    int64_t ldy;
+    // accumulator dump (parity hook); acc == nullptr in production
+    int32_t* acc;
+    int row0, rows, col0, cols;
+};
+cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st);
+cudaError_t gemm_i8_init();     // one-time function attributes (dynamic shared memory opt-in)
+
+}  // namespace rudder

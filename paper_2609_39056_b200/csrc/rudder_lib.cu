@@ -1,0 +1,9 @@
+// The library is built as ONE translation unit: the kernels share a device status word and inline
+// PTX helpers, and nothing needs relocatable device code.
+#include "internal.cuh"
+#include "ptx.cuh"
+
+#include "pack.cu"
+#include "actq.cu"
+#include "gemm_i8.cu"
+#include "api.cu"

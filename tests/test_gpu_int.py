@@ -1,0 +1,185 @@
+"""GPU parity of the integer schemes (W4A8, W4A4-INT) against the CPU oracle, through the C ABI:
+pack export, activation codes, row scales and INT32 group accumulators bit-exact; BF16 outputs
+within max relative error 1e-2 plus absolute error 2e-2 of the oracle's fp64 evaluation."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from helpers import GpuLinear, bf16_to_np, check_output, oracle_pack, static_clip, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rd():
+    import paper_2609_39056_b200 as rd
+    rd.lib()
+    return rd
+
+
+def _assert_clean(rd):
+    last, where = rd.rudder_device_status()
+    assert last == 0, f"device status {last} (wait code {where})"
+
+
+@pytest.mark.parametrize("N,K,G", [(64, 128, 64), (128, 256, 128), (256, 512, 512), (320, 1024, 64)])
+def test_pack_export_bit_exact(rd, N, K, G):
+    inp = wl.tiny(seed=100 + N, M=4, K=K, N=N)
+    ref = oracle.pack_int4(inp.W, inp.d, G)
+    g = GpuLinear(rd, inp, "w4a8", G)
+    ex = rd.rudder_weight_export(g.w)
+    assert np.array_equal(ex["codes"].cpu().numpy(), ref["packed"])
+    assert np.array_equal(ex["scales"].view(torch.int16).cpu().numpy().view(np.uint16), ref["scales"])
+    assert np.array_equal(ex["dinv"].cpu().numpy().view(np.uint32), ref["dinv"].view(np.uint32))
+    _assert_clean(rd)
+
+
+def test_pack_without_channel_scales(rd):
+    inp = wl.tiny(seed=101, M=4, K=256, N=64)
+    ref = oracle.pack_int4(inp.W, None, 64)
+    W = torch.from_numpy(inp.W).cuda()
+    w = rd.rudder_pack_weights(W, None, rd.W4A8_INT, 64)
+    ex = rd.rudder_weight_export(w)
+    assert np.array_equal(ex["codes"].cpu().numpy(), ref["packed"])
+    assert np.array_equal(ex["dinv"].cpu().numpy(), np.ones(256, np.float32))
+
+
+@pytest.mark.parametrize("scheme,qmax", [("w4a8", 127), ("w4a4", 7)])
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("M,K", [(1, 128), (37, 384), (130, 1024), (64, 2048), (19, 4096), (9, 8192), (5, 12288)])
+def test_activation_codes_bit_exact(rd, scheme, qmax, mode, M, K):
+    inp = wl.tiny(seed=200 + M, M=M, K=K, N=64, T=3)
+    ref_w = oracle.pack_int4(inp.W, inp.d, 64)
+    clip = static_clip(inp, ref_w["dinv"]) if mode == 1 else None
+    g = GpuLinear(rd, inp, scheme, 64, mode, clip)
+    for step in (0, 2):
+        codes, _, r = rd.rudder_quantize_activations(g.w, g.X, g.seg, step, g.tab)
+        rc, rr = oracle.quantize_int(inp.X_bf16, ref_w["dinv"], inp.gamma, clip, step, mode, inp.seg_offsets,
+                                     inp.seg_stream, qmax)
+        assert np.array_equal(codes.cpu().numpy(), rc)
+        assert np.array_equal(r.cpu().numpy().view(np.uint32), rr.view(np.uint32))
+    _assert_clean(rd)
+
+
+def test_activation_zero_row_and_strided_input(rd):
+    inp = wl.tiny(seed=201, M=12, K=256, N=64, T=1)
+    inp.X_bf16[3] = 0
+    ref_w = oracle.pack_int4(inp.W, inp.d, 64)
+    g = GpuLinear(rd, inp, "w4a8", 64)
+    wide = torch.zeros((12, 256 + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :256] = g.X
+    codes, _, r = rd.rudder_quantize_activations(g.w, wide[:, :256], g.seg, 0, g.tab)
+    rc, rr = oracle.quantize_int(inp.X_bf16, ref_w["dinv"], inp.gamma, None, 0, 0, inp.seg_offsets, inp.seg_stream, 127)
+    assert np.array_equal(codes.cpu().numpy(), rc) and np.array_equal(r.cpu().numpy(), rr)
+    assert r[3].item() == 0.0 and not codes[3].any().item()
+
+
+CASES = [
+    # M, K, N, G, scheme
+    (8, 128, 64, 64, "w4a8"),          # one stage, two groups, narrow ragged N tile
+    (128, 256, 128, 64, "w4a8"),
+    (130, 384, 256, 64, "w4a8"),       # ragged M tail, wide tile
+    (200, 512, 320, 128, "w4a8"),      # N = 320: 128-wide tiles with a ragged last tile
+    (64, 512, 256, 512, "w4a8"),       # G = K: the paper's per-output-channel scales (Eq. 10 verbatim)
+    (257, 1024, 512, 64, "w4a4"),
+    (96, 256, 256, 128, "w4a4"),
+    (33, 2304, 256, 64, "w4a8"),       # 18 stages: every ring wraps several times
+]
+
+
+@pytest.mark.parametrize("M,K,N,G,scheme", CASES)
+@pytest.mark.parametrize("mode", [0, 1])
+def test_linear_accumulators_and_output(rd, M, K, N, G, scheme, mode):
+    qmax = 127 if scheme == "w4a8" else 7
+    inp = wl.tiny(seed=300 + M + N, M=M, K=K, N=N, T=2)
+    ref_w = oracle.pack_int4(inp.W, inp.d, G)
+    clip = static_clip(inp, ref_w["dinv"]) if mode == 1 else None
+    g = GpuLinear(rd, inp, scheme, G, mode, clip)
+    step = 1
+    Y, acc = rd.rudder_linear_dump_acc(g.w, g.X, g.seg, step, g.tab, g.bias)
+    rc, rr = oracle.quantize_int(inp.X_bf16, ref_w["dinv"], inp.gamma, clip, step, mode, inp.seg_offsets,
+                                 inp.seg_stream, qmax)
+    racc = oracle.accumulate_int(rc, ref_w["qw"], G)
+    assert np.array_equal(acc.cpu().numpy(), racc), "INT32 group accumulators differ"
+    _, y64 = oracle.linear_int(rc, rr, ref_w["qw"], ref_w["scales"], G, inp.bias)
+    check_output(bf16_to_np(Y), y64)
+    # the production entry point (no dump) gives the same bits
+    Y2 = rd.rudder_linear(g.w, g.X, g.seg, step, g.tab, g.bias)
+    assert torch.equal(Y, Y2)
+    _assert_clean(rd)
+
+
+def test_linear_no_bias_and_padded_output(rd):
+    inp = wl.tiny(seed=301, M=70, K=256, N=128, T=1)
+    ref_w = oracle.pack_int4(inp.W, inp.d, 64)
+    g = GpuLinear(rd, inp, "w4a8", 64)
+    Ybuf = torch.full((70, 128 + 8), 7.0, dtype=torch.bfloat16, device="cuda")
+    rd.rudder_linear(g.w, g.X, g.seg, 0, g.tab, None, Y=Ybuf[:, :128])
+    out = oracle.rudder_linear(inp.X_bf16, ref_w, inp.gamma, None, 0, 0, inp.seg_offsets, inp.seg_stream, "w4a8", None)
+    check_output(bf16_to_np(Ybuf[:, :128]), out["y64"])
+    assert (Ybuf[:, 128:] == 7.0).all().item()          # nothing written past N
+    _assert_clean(rd)
+
+
+def test_config0_full(rd):
+    """Configuration 0: M = 256 (192 video / 16 proprio / 48 action), K = N = 1024, W4A8, G = 64."""
+    cfg = wl.config(0)
+    inp = cfg.draw()[0]
+    ref_w = oracle.pack_int4(inp.W, inp.d, cfg.group)
+    g = GpuLinear(rd, inp, cfg.scheme, cfg.group)
+    Y, acc = rd.rudder_linear_dump_acc(g.w, g.X, g.seg, 0, g.tab, g.bias)
+    out = oracle.rudder_linear(inp.X_bf16, ref_w, inp.gamma, None, 0, 0, inp.seg_offsets, inp.seg_stream, "w4a8", inp.bias)
+    assert np.array_equal(acc.cpu().numpy(), oracle.accumulate_int(out["codes"], ref_w["qw"], cfg.group))
+    fro, worst = check_output(bf16_to_np(Y), out["y64"])
+    assert fro < 4e-3
+    _assert_clean(rd)
+
+
+def test_row_independence_on_gpu(rd):
+    """Rows 120..135 straddle a 128-row tile and a segment boundary; a sub-call on them alone gives
+    the same bits as the full call."""
+    inp = wl.tiny(seed=302, M=256, K=512, N=256, T=1, parts=[(126, 0), (6, 1), (124, 2)])
+    g = GpuLinear(rd, inp, "w4a8", 64)
+    Y = rd.rudder_linear(g.w, g.X, g.seg, 0, g.tab, g.bias)
+    sub_seg = rd.Segments([0, 6, 12, 16], [0, 1, 2])
+    Ys = rd.rudder_linear(g.w, g.X[120:136], sub_seg, 0, g.tab, g.bias)
+    assert torch.equal(Y[120:136], Ys)
+    _assert_clean(rd)
+
+
+def test_block_matches_four_linears(rd):
+    H, F, M = 256, 512, 150
+    rng = np.random.default_rng(5)
+    so, ss = wl.segments([(100, 0), (20, 1), (30, 2)])
+    lins = [wl.draw_linear(rng, M, K, N, 2, 3, so, ss, 0.01, 30.0) for K, N in [(H, 3 * H), (H, H), (H, F), (F, H)]]
+    gs = [GpuLinear(rd, l, "w4a8", 64) for l in lins]
+    ys = [torch.empty((M, l.N), dtype=torch.bfloat16, device="cuda") for l in lins]
+    args = rd.BlockArgs([g.w for g in gs], [g.tab for g in gs], [g.bias for g in gs], [g.X for g in gs], ys)
+    ws = torch.empty(rd.rudder_block_workspace_bytes(args, M) + 256, dtype=torch.uint8, device="cuda")
+    rd.rudder_block(args, M, gs[0].seg, 1, ws)
+    for g, l, y in zip(gs, lins, ys):
+        ref_w = oracle.pack_int4(l.W, l.d, 64)
+        out = oracle.rudder_linear(l.X_bf16, ref_w, l.gamma, None, 1, 0, l.seg_offsets, l.seg_stream, "w4a8", l.bias)
+        check_output(bf16_to_np(y), out["y64"])
+        assert torch.equal(y, rd.rudder_linear(g.w, g.X, g.seg, 1, g.tab, g.bias))
+    _assert_clean(rd)
+
+
+def test_argument_errors_on_device_box(rd):
+    inp = wl.tiny(seed=303, M=16, K=128, N=64, T=2)
+    g = GpuLinear(rd, inp, "w4a8", 64)
+    with pytest.raises(rd.RudderError) as e:
+        rd.rudder_linear(g.w, g.X, g.seg, 2, g.tab, g.bias)            # step out of range
+    assert e.value.status == rd.ERR_ARG
+    with pytest.raises(rd.RudderError) as e:
+        rd.rudder_linear(g.w, g.X, rd.Segments([0, 8], [0]), 0, g.tab)  # segments do not cover M
+    assert e.value.status == rd.ERR_ARG
+    with pytest.raises(rd.RudderError) as e:
+        rd.rudder_linear(g.w, g.X, g.seg, 0, rd.ScaleTable(g.gamma, None, rd.RANGE_STATIC))   # static without clip
+    assert e.value.status == rd.ERR_ARG
+    with pytest.raises(rd.RudderError) as e:
+        rd.rudder_linear(g.w, g.X, g.seg, 0, g.tab, workspace=torch.empty(512, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == rd.ERR_WORKSPACE
+    _assert_clean(rd)

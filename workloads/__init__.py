@@ -143,9 +143,8 @@ def tiny(seed=0, M=8, K=128, N=64, T=2, S=3, parts=None, outlier_frac=0.02, outl
     """A small seeded case for brute-force checks."""
     rng = np.random.default_rng(seed)
     if parts is None:
-        a = max(1, M // 2)
-        b = max(1, (M - a) // 2)
-        parts = [(a, VIDEO), (b, PROPRIO), (M - a - b, ACTION)]
-        parts = [p for p in parts if p[0] > 0]
+        a = (M + 1) // 2
+        b = (M - a + 1) // 2
+        parts = [p for p in [(a, VIDEO), (b, PROPRIO), (M - a - b, ACTION)] if p[0] > 0]
     so, ss = segments(parts)
     return draw_linear(rng, M, K, N, T, S, so, ss, outlier_frac, outlier_gain)
