@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the fused quantized-linear hot path on B200.
+
+A "step" is one pass of the whole hot path over one batch of synthetic input: the four quantized
+linears (QKV, O, MLP-up, MLP-down) of one DiT block for one denoising step = 4 activation prologues
++ 4 low-bit GEMMs with fused epilogue (rudder_block).  Default workload: configuration 2 (W4A8,
+hidden 2048, MLP 8192, 4096 video + 64 proprio + 256 action tokens, group 64, 10 steps of tables).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg3_nvfp4] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded row sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "fused W4A8/W4A4 DiT-block linear chain throughput (2*M*K*N over QKV, O, up, down per step)"
+UNIT = "TOPS"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def workload_config(name: str):
+    if name == "cfg2":
+        return wl.config(2)
+    if name == "cfg3":
+        return wl.config(3, "w4a4")
+    if name == "cfg3_nvfp4":
+        return wl.config(3, "nvfp4")
+    raise SystemExit(f"unknown workload {name}")
+
+
+def algorithmic_bytes_linear(M, K, N, G, scheme):
+    """Bytes one linear must move in the two-kernel form: X, codes + r written then read, packed W +
+    scales, Y, bias."""
+    if scheme == "nvfp4":
+        act = M * K // 2 + M * K // 16 + 4 * M
+        w = N * K // 2 + N * K // 16 + 4
+    else:
+        act = M * K + 4 * M           # one code per byte in the workspace (both integer schemes)
+        w = N * K // 2 + 2 * N * K // G
+    return 2 * M * K + 2 * act + w + 2 * M * N + 4 * N
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 100 ms in the background."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0, t1):
+        sm, smax, reasons = [], 0.0, set()
+        for t, line in self.samples:
+            if t < t0 or t > t1:
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax = max(smax, float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return None
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": smax, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_block(rd, cfg, torch, dev):
+    """Pack the four weights and put the replay inputs of one block on the device."""
+    lins = cfg.draw()
+    scheme = rd.SCHEMES[cfg.scheme]
+    ws, tabs, biases, xs, ys, keep = [], [], [], [], [], []
+    for l in lins:
+        W = torch.from_numpy(l.W).to(dev)
+        d = torch.from_numpy(l.d).to(dev)
+        ws.append(rd.rudder_pack_weights(W, d, scheme, cfg.group))
+        del W, d
+        gamma = torch.from_numpy(l.gamma).to(dev)
+        tabs.append(rd.ScaleTable(gamma, None, rd.RANGE_PER_TOKEN))
+        biases.append(torch.from_numpy(l.bias).to(dev))
+        xs.append(torch.from_numpy(l.X_bf16.view(np.int16)).to(dev).view(torch.bfloat16))
+        ys.append(torch.empty((l.M, l.N), dtype=torch.bfloat16, device=dev))
+    seg = rd.Segments(lins[0].seg_offsets, lins[0].seg_stream)
+    return lins, ws, tabs, biases, xs, ys, seg
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    import paper_2609_39056_b200 as rd
+    rd.lib()
+
+    cfg = workload_config(args.workload)
+    M, T = cfg.M, cfg.T
+    lins, ws, tabs, biases, xs, ys, seg = build_block(rd, cfg, torch, dev)
+    bargs = rd.BlockArgs(ws, tabs, biases, xs, ys)
+    workspace = torch.empty(rd.rudder_block_workspace_bytes(bargs, M) + 256, dtype=torch.uint8, device=dev)
+    ops = cfg.ops()
+    alg_bytes = [algorithmic_bytes_linear(M, K, N, cfg.group, cfg.scheme) for _, K, N in cfg.linears]
+    launches_per_step = 8
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: K steps bracketed by barrier + synchronize, CUDA events on the launch stream
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    for i in range(args.warmup):
+        rd.rudder_block(bargs, M, seg, i % T, workspace)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t_wall0 = time.time()
+    ev0.record()
+    for i in range(args.steps):
+        rd.rudder_block(bargs, M, seg, i % T, workspace)
+    ev1.record()
+    barrier()
+    t_wall1 = time.time()
+    ms_total = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * ops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- clocks under this load (repeat the same steps if the timed region was too short to sample)
+    clocks = None
+    if rank == 0:
+        clocks = sampler.summary(t_wall0, t_wall1)
+        if clocks is None or clocks["samples"] < 3:
+            t0 = time.time()
+            while time.time() - t0 < 1.5:
+                for i in range(50):
+                    rd.rudder_block(bargs, M, seg, i % T, workspace)
+                torch.cuda.synchronize()
+            clocks = sampler.summary(t0, time.time())
+            if clocks is not None:
+                clocks["note"] = "timed region shorter than the sampling period: sampled while replaying the same steps for 1.5 s"
+        sampler.stop()
+    status, where = rd.rudder_device_status()
+    if status != 0:
+        raise SystemExit(f"device status {status} (wait {where}): the run is invalid")
+
+    # ---- per-kernel times (events between launches) for the roofline of the dominant kernel
+    prof = np.zeros(8)
+    n_prof = max(3, min(10, args.steps))
+    for i in range(n_prof):
+        prof += np.array(rd.rudder_block_profile(bargs, M, seg, i % T, workspace))
+    prof /= n_prof
+    gemm_ms = float(prof[1::2].sum())
+    actq_ms = float(prof[0::2].sum())
+    pk = peaks()
+    int8_peak = 2.0 * pk["bf16_sustained"]        # kind::i8 runs at twice the bf16 rate
+    fp4_peak = 4.0 * pk["bf16_sustained"]
+    tensor_peak = fp4_peak if cfg.scheme == "nvfp4" else int8_peak
+    achieved = ops / (gemm_ms * 1e-3) / 1e12
+    roofline = {"kernel": "gemm (4 launches per step)", "bound": "tensor", "achieved": achieved, "peak": tensor_peak,
+                "unit": "TOPS" if cfg.scheme != "nvfp4" else "TFLOP/s", "frac": achieved / tensor_peak,
+                "peak_source": f"{pk['source']} bf16 sustained x {'4' if cfg.scheme == 'nvfp4' else '2'} (nominal ratio)",
+                "traffic": None, "gemm_ms": gemm_ms, "prologue_ms": actq_ms,
+                "prologue_hbm_gbs": sum((2 * M * K + M * K + 4 * M) for _, K, N in cfg.linears) / (actq_ms * 1e-3) / 1e9,
+                "prologue_hbm_frac": sum((2 * M * K + M * K + 4 * M) for _, K, N in cfg.linears) / (actq_ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                "per_kernel_ms": [float(v) for v in prof]}
+
+    # ---- end to end through the C ABI with HOST buffers (pinned): H2D of the 4 inputs, block, D2H of the 4 outputs
+    hx = [x.cpu().pin_memory() for x in xs]
+    hy = [torch.empty(y.shape, dtype=y.dtype).pin_memory() for y in ys]
+    hargs = rd.BlockArgs(ws, tabs, biases, hx, hy)
+    staging = torch.empty(rd.rudder_block_host_staging_bytes(hargs, M) + 256, dtype=torch.uint8, device=dev)
+    e2e_steps = max(3, min(args.steps, 20))
+    for i in range(2):
+        rd.rudder_block_host(hargs, M, seg, i % T, staging, workspace)
+    barrier()
+    ev0.record()
+    for i in range(e2e_steps):
+        rd.rudder_block_host(hargs, M, seg, i % T, staging, workspace)
+    ev1.record()
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(int(x.numel()) * 2 for x in hx)
+    d2h = sum(int(y.numel()) * 2 for y in hy)
+    e2e = {"value": world * ops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- cuBLAS BF16 on the same shapes (speed-up reference only)
+    bf16_ms = None
+    if rank == 0 and not args.no_bf16:
+        wbf = [torch.randn((N, K), dtype=torch.bfloat16, device=dev) for _, K, N in cfg.linears]
+        for _ in range(3):
+            for x, w_ in zip(xs, wbf):
+                torch.matmul(x, w_.t())
+        torch.cuda.synchronize()
+        ev0.record()
+        reps = 10
+        for _ in range(reps):
+            for x, w_ in zip(xs, wbf):
+                torch.matmul(x, w_.t())
+        ev1.record()
+        torch.cuda.synchronize()
+        bf16_ms = ev0.elapsed_time(ev1) / reps
+        del wbf
+
+    # ---- the oracle on this machine's host cores, on a bounded row sample (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline(cfg, lins, target_s=args.cpu_seconds)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "us_per_block_step": ms_per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": {"w4a8": "int8 x int4 -> int32", "w4a4": "int4 x int4 -> int32",
+                                                              "nvfp4": "e2m1 x e2m1 -> fp32"}[cfg.scheme],
+            "data": "synthetic", "gpu_launches": launches_per_step * args.steps,
+            "config": {"workload": cfg.name, "scheme": cfg.scheme, "group": cfg.group, "M": M,
+                       "linears": {n: [K, N] for n, K, N in cfg.linears}, "range_mode": "per_token",
+                       "steps_of_tables": T, "tops_per_step": ops / 1e12,
+                       "l2": f"working set per step {sum(alg_bytes) / 1e6:.0f} MB (inputs {sum(2 * M * K for _, K, _ in cfg.linears) / 1e6:.0f} MB) exceeds the 126 MB L2; no explicit flush",
+                       "parallelism": f"replicas x{world} (rows independent, no collective)"},
+            "clocks": clocks, "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu,
+            "bf16_cublas_ms_per_step": bf16_ms,
+            "speedup_vs_bf16_cublas": (bf16_ms / ms_per_step) if bf16_ms else None,
+            "algorithmic_mb_per_step": sum(alg_bytes) / 1e6,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(cfg, lins, target_s=15.0, impl_reference=False):
+    """Time the oracle, as it stands, on a bounded sample of rows of the same workload."""
+    import oracle
+    cores = oracle.num_threads()
+    packs = []
+    for l in lins:
+        packs.append(oracle.pack_nvfp4(l.W, l.d) if cfg.scheme == "nvfp4" else oracle.pack_int4(l.W, l.d, cfg.group))
+    M = cfg.M
+
+    def run(rows):
+        t0 = time.time()
+        for l, pw in zip(lins, packs):
+            oracle.rudder_linear(l.X_bf16, pw, l.gamma, None, 0, oracle.RANGE_PER_TOKEN, l.seg_offsets, l.seg_stream,
+                                 cfg.scheme, l.bias, rows=rows)
+        return time.time() - t0
+
+    rng = np.random.default_rng(1234)
+    n0 = min(M, 4 * cores)
+    t_probe = run(np.sort(rng.choice(M, n0, replace=False)).astype(np.int32))
+    n = int(min(M, max(n0, n0 * target_s / max(t_probe, 1e-3))))
+    n = max(cores, n // cores * cores)
+    rows = np.sort(rng.choice(M, n, replace=False)).astype(np.int32)
+    t = run(rows)
+    ops_sample = sum(2.0 * n * K * N for _, K, N in cfg.linears)
+    return {"value": ops_sample / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{n} of {M} rows (seeded), all four linears, step 0, {t:.1f} s wall", "seconds": t}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on this machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = workload_config(args.workload)
+    lins = cfg.draw()
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    res = None
+    times = []
+    for i in range(args.warmup + args.steps):
+        res = cpu_baseline(cfg, lins, target_s=per_step)
+        if i >= args.warmup:
+            times.append(res["value"])
+    value = float(np.mean(times))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": res["seconds"] * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "oracle (fp32 / int32 / fp64 on CPU)", "data": "synthetic",
+            "config": {"workload": cfg.name, "scheme": cfg.scheme, "group": cfg.group, "M": cfg.M,
+                       "linears": {n: [K, N] for n, K, N in cfg.linears}},
+            "cpu_baseline": {"kind": "oracle", "cores": res["cores"], "sample": res["sample"], "value": value, "unit": UNIT},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
+    ap.add_argument("--no-bf16", action="store_true", help="skip the cuBLAS BF16 comparison")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -138,6 +138,22 @@ size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M);
 rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* Measurement hook: rudder_block with a CUDA event between consecutive kernels.  ms (HOST [8])
+ * receives the device time of each launch in order: prologue and GEMM of QKV, O, up, down.
+ * Creates and destroys its events and SYNCHRONISES the stream before returning. */
+rudder_status rudder_block_profile(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
+                                   void* workspace, size_t workspace_bytes, void* stream, float* ms);
+
+/* rudder_block for callers whose activations live in HOST memory (pinned for asynchronous copies):
+ * args->x[l] and args->y[l] are HOST pointers here (rows contiguous: ldx[l] >= K_l, ldy[l] >= N_l);
+ * everything else is as in rudder_block.  Each input is copied to `staging`, the block runs, each
+ * output is copied back, all on `stream`, without synchronising.  staging: device memory of at
+ * least rudder_block_host_staging_bytes(args, M) bytes, 256-byte aligned. */
+size_t rudder_block_host_staging_bytes(const rudder_block_args* args, int M);
+rudder_status rudder_block_host(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
+                                void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,
+                                void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Parity hooks: the production kernels, with their intermediate results written in canonical form.
  */

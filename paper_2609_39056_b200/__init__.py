@@ -24,6 +24,7 @@ SCHEMES = {"w4a8": W4A8_INT, "w4a4": W4A4_INT, "nvfp4": W4A4_NVFP4}
 EXPORTED = [
     "rudder_pack_weights", "rudder_weight_free", "rudder_weight_info", "rudder_weight_export",
     "rudder_linear_workspace_bytes", "rudder_linear", "rudder_block_workspace_bytes", "rudder_block",
+    "rudder_block_profile", "rudder_block_host_staging_bytes", "rudder_block_host",
     "rudder_quantize_activations", "rudder_linear_dump_acc", "rudder_device_status", "rudder_status_string",
 ]
 
@@ -76,6 +77,11 @@ def lib() -> ctypes.CDLL:
         L.rudder_block_workspace_bytes.restype = sz
         L.rudder_block_workspace_bytes.argtypes = [ctypes.POINTER(_BlockArgs), i32]
         L.rudder_block.argtypes = [ctypes.POINTER(_BlockArgs), i32, ctypes.POINTER(_Segments), i32, vp, sz, vp]
+        L.rudder_block_profile.argtypes = [ctypes.POINTER(_BlockArgs), i32, ctypes.POINTER(_Segments), i32, vp, sz, vp,
+                                           ctypes.POINTER(ctypes.c_float)]
+        L.rudder_block_host_staging_bytes.restype = sz
+        L.rudder_block_host_staging_bytes.argtypes = [ctypes.POINTER(_BlockArgs), i32]
+        L.rudder_block_host.argtypes = [ctypes.POINTER(_BlockArgs), i32, ctypes.POINTER(_Segments), i32, vp, sz, vp, sz, vp]
         L.rudder_quantize_activations.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32,
                                                   ctypes.POINTER(_ScaleTable), vp, vp, vp, vp]
         L.rudder_linear_dump_acc.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32,
@@ -255,6 +261,28 @@ def rudder_block(args: BlockArgs, M: int, seg: Segments, step: int, workspace: t
     wp, wb = _aligned(workspace)
     _check(lib().rudder_block(ctypes.byref(args.c), int(M), ctypes.byref(seg.c), int(step), wp, wb, _stream(stream)),
            "rudder_block")
+
+
+def rudder_block_profile(args: BlockArgs, M: int, seg: Segments, step: int, workspace: torch.Tensor, stream=None):
+    """rudder_block with an event between kernels -> 8 device times in ms (prologue, GEMM) x (QKV, O, up, down)."""
+    wp, wb = _aligned(workspace)
+    ms = (ctypes.c_float * 8)()
+    _check(lib().rudder_block_profile(ctypes.byref(args.c), int(M), ctypes.byref(seg.c), int(step), wp, wb,
+                                      _stream(stream), ms), "rudder_block_profile")
+    return [float(v) for v in ms]
+
+
+def rudder_block_host_staging_bytes(args: BlockArgs, M: int) -> int:
+    return int(lib().rudder_block_host_staging_bytes(ctypes.byref(args.c), int(M)))
+
+
+def rudder_block_host(args: BlockArgs, M: int, seg: Segments, step: int, staging: torch.Tensor,
+                      workspace: torch.Tensor, stream=None):
+    """rudder_block whose x / y tensors in ``args`` are (pinned) HOST tensors."""
+    sp, sb = _aligned(staging)
+    wp, wb = _aligned(workspace)
+    _check(lib().rudder_block_host(ctypes.byref(args.c), int(M), ctypes.byref(seg.c), int(step), sp, sb, wp, wb,
+                                   _stream(stream)), "rudder_block_host")
 
 
 def rudder_device_status():

@@ -100,7 +100,7 @@ size_t workspace_bytes_for(const rudder_weight* w, int M)
 rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M, const rudder_segments* seg,
                           int step, const rudder_scale_table* tab, const float* bias, uint16_t* Y, int64_t ldy,
                           void* workspace, size_t workspace_bytes, cudaStream_t st, int32_t* acc, int row0, int rows,
-                          int col0, int cols)
+                          int col0, int cols, cudaEvent_t* ev = nullptr /* ev[1] recorded after the prologue, ev[2] after the GEMM */)
 {
     if (!w || !X || !Y) return RUDDER_ERR_ARG;
     if (M < 1) return RUDDER_ERR_SHAPE;
@@ -127,6 +127,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;
     a.seg = sp;
     if (launch_actq_int(a, qmax_of(w->scheme), codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
 
     GemmI8Args g;
     if (!make_tmap_2d(&g.tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(M),
@@ -137,6 +138,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     g.row_scale = r; g.bias = bias; g.Y = Y; g.ldy = ldy;
     g.acc = acc; g.row0 = row0; g.rows = rows; g.col0 = col0; g.cols = cols;
     if (launch_gemm_i8(g, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return RUDDER_ERR_CUDA;
     return RUDDER_OK;
 }
 
@@ -283,8 +285,8 @@ size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M)
     return total;
 }
 
-rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_segments* seg, int step, void* workspace,
-                           size_t workspace_bytes, void* stream)
+static rudder_status block_impl(const rudder_block_args* args, int M, const rudder_segments* seg, int step, void* workspace,
+                                size_t workspace_bytes, void* stream, cudaEvent_t* ev /* [9] or nullptr */)
 {
     if (!args) return RUDDER_ERR_ARG;
     for (int l = 0; l < 4; ++l)
@@ -304,10 +306,93 @@ rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_se
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     for (int l = 0; l < 4; ++l) {
         const size_t bytes = workspace_bytes_for(args->w[l], M);
-        rudder_status s = rudder_linear(args->w[l], args->x[l], args->ldx[l], M, seg, step, args->tab[l], args->bias[l],
-                                        args->y[l], args->ldy[l], ws, bytes, stream);
+        rudder_status s = linear_impl(args->w[l], args->x[l], args->ldx[l], M, seg, step, args->tab[l], args->bias[l],
+                                      args->y[l], args->ldy[l], ws, bytes, static_cast<cudaStream_t>(stream), nullptr, 0, 0,
+                                      0, 0, ev ? ev + 2 * l : nullptr);
         if (s != RUDDER_OK) return s;
         ws += bytes;
+    }
+    return RUDDER_OK;
+}
+
+rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_segments* seg, int step, void* workspace,
+                           size_t workspace_bytes, void* stream)
+{
+    return block_impl(args, M, seg, step, workspace, workspace_bytes, stream, nullptr);
+}
+
+rudder_status rudder_block_profile(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
+                                   void* workspace, size_t workspace_bytes, void* stream, float* ms)
+{
+    if (!ms) return RUDDER_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaEvent_t ev[9];
+    for (int i = 0; i < 9; ++i)
+        if (cudaEventCreate(&ev[i]) != cudaSuccess) return RUDDER_ERR_CUDA;
+    rudder_status s = RUDDER_OK;
+    if (cudaEventRecord(ev[0], st) != cudaSuccess) s = RUDDER_ERR_CUDA;
+    if (s == RUDDER_OK) s = block_impl(args, M, seg, step, workspace, workspace_bytes, stream, ev);
+    if (s == RUDDER_OK && cudaStreamSynchronize(st) != cudaSuccess) s = RUDDER_ERR_CUDA;
+    if (s == RUDDER_OK)
+        for (int i = 0; i < 8; ++i)
+            if (cudaEventElapsedTime(&ms[i], ev[i], ev[i + 1]) != cudaSuccess) s = RUDDER_ERR_CUDA;
+    for (int i = 0; i < 9; ++i) cudaEventDestroy(ev[i]);
+    return s;
+}
+
+size_t rudder_block_host_staging_bytes(const rudder_block_args* args, int M)
+{
+    if (!args || M < 1) return 0;
+    size_t total = 0;
+    for (int l = 0; l < 4; ++l) {
+        if (!args->w[l]) return 0;
+        total += align_up(static_cast<size_t>(M) * args->w[l]->K * 2, 256) + align_up(static_cast<size_t>(M) * args->w[l]->N * 2, 256);
+    }
+    return total;
+}
+
+rudder_status rudder_block_host(const rudder_block_args* args, int M, const rudder_segments* seg, int step, void* staging,
+                                size_t staging_bytes, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!args) return RUDDER_ERR_ARG;
+    for (int l = 0; l < 4; ++l)
+        if (!args->w[l] || !args->x[l] || !args->y[l] || args->ldx[l] < args->w[l]->K || args->ldy[l] < args->w[l]->N)
+            return RUDDER_ERR_ARG;
+    const size_t need = rudder_block_host_staging_bytes(args, M);
+    if (!staging || !aligned(staging, 256) || staging_bytes < need || need == 0) return RUDDER_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rudder_block_args dev = *args;
+    uint8_t* p = static_cast<uint8_t*>(staging);
+    for (int l = 0; l < 4; ++l) {
+        const int K = args->w[l]->K, N = args->w[l]->N;
+        dev.x[l] = reinterpret_cast<const uint16_t*>(p);
+        dev.ldx[l] = K;
+        p += align_up(static_cast<size_t>(M) * K * 2, 256);
+        dev.y[l] = reinterpret_cast<uint16_t*>(p);
+        dev.ldy[l] = N;
+        p += align_up(static_cast<size_t>(M) * N * 2, 256);
+    }
+    // validate on the host before the first copy is enqueued (block_impl checks again)
+    for (int l = 0; l < 4; ++l) {
+        SegParams sp;
+        if (!args->tab[l]) return RUDDER_ERR_ARG;
+        rudder_status s = check_table_and_segments(seg, step, args->tab[l], M, &sp);
+        if (s != RUDDER_OK) return s;
+    }
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < rudder_block_workspace_bytes(args, M)) return RUDDER_ERR_WORKSPACE;
+    for (int l = 0; l < 4; ++l) {
+        const int K = args->w[l]->K;
+        if (cudaMemcpy2DAsync(const_cast<uint16_t*>(dev.x[l]), static_cast<size_t>(K) * 2, args->x[l], static_cast<size_t>(args->ldx[l]) * 2,
+                              static_cast<size_t>(K) * 2, M, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return RUDDER_ERR_CUDA;
+    }
+    rudder_status s = block_impl(&dev, M, seg, step, workspace, workspace_bytes, stream, nullptr);
+    if (s != RUDDER_OK) return s;
+    for (int l = 0; l < 4; ++l) {
+        const int N = args->w[l]->N;
+        if (cudaMemcpy2DAsync(args->y[l], static_cast<size_t>(args->ldy[l]) * 2, dev.y[l], static_cast<size_t>(N) * 2,
+                              static_cast<size_t>(N) * 2, M, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return RUDDER_ERR_CUDA;
     }
     return RUDDER_OK;
 }
