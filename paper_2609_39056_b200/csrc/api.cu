@@ -84,11 +84,6 @@ rudder_status check_table_and_segments(const rudder_segments* seg, int step, con
 
 int qmax_of(int scheme) { return scheme == RUDDER_W4A8_INT ? 127 : 7; }
 
-struct LinearPlan {
-    SegParams seg;
-    size_t off_codes, off_r, bytes;
-};
-
 size_t workspace_bytes_for(const rudder_weight* w, int M)
 {
     if (!w || M < 1) return 0;
@@ -130,12 +125,18 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
 
     GemmI8Args g;
-    if (!make_tmap_2d(&g.tm_a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(M),
-                      static_cast<uint64_t>(w->K), 128, static_cast<uint32_t>(M < 128 ? M : 128), CU_TENSOR_MAP_SWIZZLE_128B))
+    const int tt = gemm_i8_token_tile(M);
+    const uint32_t box_tok = static_cast<uint32_t>(M < tt ? M : tt);
+    if (!make_tmap_2d(&g.tm_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(M),
+                      static_cast<uint64_t>(w->K), 128, box_tok, CU_TENSOR_MAP_SWIZZLE_128B))
         return RUDDER_ERR_CUDA;
-    g.wt = w->tiles;
+    if (!make_tmap_2d(&g.tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, static_cast<uint64_t>(w->N), static_cast<uint64_t>(M),
+                      static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128), box_tok,
+                      CU_TENSOR_MAP_SWIZZLE_NONE))
+        return RUDDER_ERR_CUDA;
+    g.w_codes = w->codes; g.w_scales_t = w->scales_t;
     g.M = M; g.N = w->N; g.K = w->K; g.G = w->G;
-    g.row_scale = r; g.bias = bias; g.Y = Y; g.ldy = ldy;
+    g.row_scale = r; g.bias = bias;
     g.acc = acc; g.row0 = row0; g.rows = rows; g.col0 = col0; g.cols = cols;
     if (launch_gemm_i8(g, st) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return RUDDER_ERR_CUDA;
@@ -194,18 +195,6 @@ rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, 
              cudaStreamSynchronize(st) == cudaSuccess;
     }
     if (tmp) cudaFree(tmp);
-    if (ok) {
-        for (int t = 0; t < 2 && ok; ++t) {
-            const int nt = t == 0 ? 128 : 256;
-            w->tiles[t].n_tile = nt;
-            const uint32_t box_rows = static_cast<uint32_t>(N < nt ? N : nt);
-            ok = make_tmap_2d(&w->tiles[t].codes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w->codes, static_cast<uint64_t>(K / 2),
-                              static_cast<uint64_t>(N), static_cast<uint64_t>(K / 2), 64, box_rows, CU_TENSOR_MAP_SWIZZLE_NONE) &&
-                 make_tmap_2d(&w->tiles[t].scales, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, w->scales_t, static_cast<uint64_t>(N),
-                              static_cast<uint64_t>(n_groups), static_cast<uint64_t>(N) * sizeof(float), box_rows, 1,
-                              CU_TENSOR_MAP_SWIZZLE_NONE);
-        }
-    }
     if (!ok) {
         rudder_weight_free(w);
         return RUDDER_ERR_CUDA;

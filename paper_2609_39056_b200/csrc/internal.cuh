@@ -31,11 +31,6 @@ struct SegParams {
 //   sf_tiled  NVFP4: UE4M3 scale factors in the tensor core's tiled order:
 //             [N/128][K/64][32 lanes][4 row-quarters][4 blocks] bytes.
 //   dinv      fp32 [K]
-struct WeightTiles {
-    CUtensorMap codes;    // packed codes, box = {64 bytes, n_tile rows}
-    CUtensorMap scales;   // scales_t, box = {n_tile floats, 1 group}
-    int n_tile;
-};
 }  // namespace rudder
 
 struct rudder_weight {
@@ -48,7 +43,6 @@ struct rudder_weight {
     float* dinv;
     float* tensor_scale;      // device [1]
     size_t bytes;
-    rudder::WeightTiles tiles[2];   // [0]: n_tile = 128, [1]: n_tile = 256
 };
 
 namespace rudder {
@@ -72,17 +66,18 @@ cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* c
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);
 
 struct GemmI8Args {
-    CUtensorMap tm_a;           // activation codes int8 [M, K], box {128, 128}, 128-byte swizzle
-    const WeightTiles* wt;
+    CUtensorMap tm_x;           // activation codes int8 [M, K], box {128 bytes, token tile}, 128-byte swizzle
+    CUtensorMap tm_y;           // output bf16 [M, N] (row pitch ldy), box {min(128, N) channels, token tile}
+    const uint8_t* w_codes;     // packed INT4 weights
+    const float* w_scales_t;    // [K/G][N]
     int M, N, K, G;
     const float* row_scale;     // r [M]
     const float* bias;          // [N] or nullptr
-    uint16_t* Y;
-    int64_t ldy;
     // accumulator dump (parity hook); acc == nullptr in production
     int32_t* acc;
     int row0, rows, col0, cols;
 };
+int gemm_i8_token_tile(int M);  // tokens per CTA tile the GEMM will use for M rows (sizes the TMA boxes)
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st);
 cudaError_t gemm_i8_init();     // one-time function attributes (dynamic shared memory opt-in)
 

@@ -14,13 +14,7 @@ namespace rudder {
 // [0] = last error (0 = none), [1] = code of the wait that gave up.
 __device__ int g_device_status[2] = {0, 0};
 
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // a wait that lasts one second is declared dead
-
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
+constexpr long long kWaitLimitCycles = 2000000000ll;   // a wait of ~1 s of SM clocks is declared dead
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -53,15 +47,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  `abort_word` is a shared int: non-zero means some role of this CTA gave up.
+// `sleep_ns` > 0: back off between polls so that a waiting warp does not take issue slots from the
+// warps that share its scheduler.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int where) {
-    unsigned long long t0 = 0;
-    for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();          // SM-local cycle counter: cheap to read
+    for (uint32_t it = 1;; ++it) {
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
+        if ((it & 255u) == 0u) {
             if (*abort_word != 0) return false;
-            const unsigned long long now = global_timer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) break;
+            if (clock64() - t0 > kWaitLimitCycles) break;
         }
     }
     *abort_word = where;
@@ -76,6 +73,19 @@ template <int N> __device__ __forceinline__ void reg_dec() {
 }
 template <int N> __device__ __forceinline__ void reg_inc() {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// One lane of a converged warp (the same lane every time it is called with a full mask).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t is_leader;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(is_leader));
+    return is_leader != 0;
 }
 
 // ---- proxies / fences ----------------------------------------------------------------------
