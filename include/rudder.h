@@ -118,6 +118,26 @@ rudder_status rudder_linear(const rudder_weight* w, const uint16_t* X, int64_t l
                             const float* bias, uint16_t* Y, int64_t ldy,
                             void* workspace, size_t workspace_bytes, void* stream);
 
+/* rudder_linear_static -- rudder_linear without a caller-supplied workspace.  (The paper has no
+ * counterpart: this is a convenience of this library.)
+ * For callers that cannot allocate device memory -- code inside a captured or real-time region where
+ * cudaMalloc is off limits, plug-ins that only receive input and output buffers, hosts whose memory
+ * pool belongs to another component.  Q_X and r are kept in a fixed array of
+ * rudder_linear_static_max_workspace_bytes() = 4 MiB that is part of the library image (every GPU
+ * that loads the library holds it until the process exits).  The call allocates nothing.
+ *   - Same arguments, results and errors as rudder_linear, minus the workspace.  If
+ *     rudder_linear_workspace_bytes(w, M) exceeds the 4 MiB array the call returns
+ *     RUDDER_ERR_WORKSPACE and launches nothing.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; nothing
+ *     in it needs clearing between calls.  Two calls whose kernels may overlap on the GPU (different
+ *     streams, or concurrent host threads) race on it: serialise them. */
+size_t rudder_linear_static_max_workspace_bytes(void);
+rudder_status rudder_linear_static(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M,
+                                   const rudder_segments* seg, int step, const rudder_scale_table* tab,
+                                   const float* bias, uint16_t* Y, int64_t ldy, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * rudder_block -- the four quantized linears of one DiT block for one denoising step, replaying
  * caller-supplied inputs (the paper times DiT replay with captured inputs; attention, norms and

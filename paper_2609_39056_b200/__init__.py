@@ -24,6 +24,7 @@ SCHEMES = {"w4a8": W4A8_INT, "w4a4": W4A4_INT, "nvfp4": W4A4_NVFP4}
 EXPORTED = [
     "rudder_pack_weights", "rudder_weight_free", "rudder_weight_info", "rudder_weight_export",
     "rudder_linear_workspace_bytes", "rudder_linear", "rudder_block_workspace_bytes", "rudder_block",
+    "rudder_linear_static_max_workspace_bytes", "rudder_linear_static",
     "rudder_block_profile", "rudder_block_host_staging_bytes", "rudder_block_host",
     "rudder_quantize_activations", "rudder_linear_dump_acc", "rudder_device_status", "rudder_status_string",
 ]
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.rudder_linear_workspace_bytes.argtypes = [vp, i32]
         L.rudder_linear.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32, ctypes.POINTER(_ScaleTable),
                                     vp, vp, i64, vp, sz, vp]
+        L.rudder_linear_static_max_workspace_bytes.restype = sz
+        L.rudder_linear_static_max_workspace_bytes.argtypes = []
+        L.rudder_linear_static.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32, ctypes.POINTER(_ScaleTable),
+                                           vp, vp, i64, vp]
         L.rudder_block_workspace_bytes.restype = sz
         L.rudder_block_workspace_bytes.argtypes = [ctypes.POINTER(_BlockArgs), i32]
         L.rudder_block.argtypes = [ctypes.POINTER(_BlockArgs), i32, ctypes.POINTER(_Segments), i32, vp, sz, vp]
@@ -201,6 +206,25 @@ def rudder_linear(w: Weight, X: torch.Tensor, seg: Segments, step: int, tab: Sca
     wp, wb = _aligned(workspace)
     _check(lib().rudder_linear(w.handle, _ptr(X), X.stride(0), M, ctypes.byref(seg.c), int(step), ctypes.byref(tab.c),
                                _ptr(bias), _ptr(Y), Y.stride(0), wp, wb, _stream(stream)), "rudder_linear")
+    return Y
+
+
+def rudder_linear_static_max_workspace_bytes() -> int:
+    return int(lib().rudder_linear_static_max_workspace_bytes())
+
+
+def rudder_linear_static(w: Weight, X: torch.Tensor, seg: Segments, step: int, tab: ScaleTable, bias=None, Y=None,
+                         stream=None) -> torch.Tensor:
+    """rudder_linear for callers that cannot allocate: the scratch between the two kernels is a fixed
+    4 MiB array inside the library, so only inputs and the output are passed.  Raises
+    RudderError(ERR_WORKSPACE) when the layer needs more scratch than the array holds.  Calls that may
+    overlap on the GPU share the array and must be serialised by the caller."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M = X.shape[0]
+    assert Y is not None, "the caller passes the output buffer: this entry point allocates nothing"
+    _check(lib().rudder_linear_static(w.handle, _ptr(X), X.stride(0), M, ctypes.byref(seg.c), int(step),
+                                      ctypes.byref(tab.c), _ptr(bias), _ptr(Y), Y.stride(0), _stream(stream)),
+           "rudder_linear_static")
     return Y
 
 

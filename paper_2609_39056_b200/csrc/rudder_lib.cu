@@ -7,3 +7,4 @@
 #include "actq.cu"
 #include "gemm_i8.cu"
 #include "api.cu"
+#include "static_ws.cu"
