@@ -8,6 +8,7 @@
 // second time, from L2).  All fp32 operations are individually rounded, in the order
 // v = (x * dinv) * gamma, q = rint(v * (q_max / a)), r = (a / q_max) / gamma.
 #include "internal.cuh"
+#include "fp4.cuh"
 
 namespace rudder {
 
@@ -126,6 +127,118 @@ __global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int
     }
     if (lane == 0)
         r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, static_cast<float>(qmax)), g) : 0.0f;
+}
+
+// ---- NVFP4 activations -------------------------------------------------------------------------
+// One warp per row; a lane owns one block of 16 channels per step (two 16-byte loads), so a warp step
+// covers 512 channels.  Writes packed E2M1 codes [M, K/2], one UE4M3 scale per block (in the tensor
+// core's tiled order, or row-major for the parity hook) and the row scale r = (a / 2688) / gamma.
+// Rows in [M, M_pad) only get zero scales, so that the GEMM never reads uninitialised scale bytes.
+__device__ __forceinline__ void scale16(const uint4& x0, const uint4& x1, const float4* dv, float g, float (&v)[16]) {
+    float a[8], b[8];
+    scale8(x0, __ldg(dv), __ldg(dv + 1), g, a);
+    scale8(x1, __ldg(dv + 2), __ldg(dv + 3), g, b);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { v[i] = a[i]; v[8 + i] = b[i]; }
+}
+
+template <int NIT>
+__global__ void __launch_bounds__(256) actq_nvfp4_kernel(ActqArgs a, int M_pad, uint8_t* __restrict__ codes,
+                                                          uint8_t* __restrict__ sf, int sf_tiled, float* __restrict__ r)
+{
+    const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= M_pad) return;
+    const int n_blocks = a.K >> 4;                 // 16-channel blocks in the row
+    const int n_it = (n_blocks + 31) >> 5;
+    const int k64 = a.K >> 6;
+    if (row >= a.M) {                              // padding row of the last 128-row scale atom
+        for (int kb = lane; kb < n_blocks; kb += 32) sf[nvfp4_sf_offset(row, kb, k64)] = 0;
+        return;
+    }
+    const float g = a.gamma_step[stream_of_row(a.seg, row)];
+    const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(row) * a.ldx);
+    const float4* dv = reinterpret_cast<const float4*>(a.dinv);
+
+    uint4 xr[NIT > 0 ? 2 * NIT : 2];
+    float amax = 0.0f;
+    if (NIT > 0) {
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int kb = it * 32 + lane;
+            if (kb < n_blocks) { xr[2 * it] = ld_nc_16(xrow + 2 * kb); xr[2 * it + 1] = ld_nc_16(xrow + 2 * kb + 1); }
+        }
+    }
+    if (a.clip_step == nullptr) {
+        if (NIT > 0) {
+#pragma unroll
+            for (int it = 0; it < NIT; ++it) {
+                const int kb = it * 32 + lane;
+                if (kb < n_blocks) {
+                    float v[16];
+                    scale16(xr[2 * it], xr[2 * it + 1], dv + 4 * kb, g, v);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+                }
+            }
+        } else {
+            for (int it = 0; it < n_it; ++it) {
+                const int kb = it * 32 + lane;
+                if (kb < n_blocks) {
+                    float v[16];
+                    scale16(ld_nc_16(xrow + 2 * kb), ld_nc_16(xrow + 2 * kb + 1), dv + 4 * kb, g, v);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    }
+    const float range = a.clip_step ? *a.clip_step : amax;
+    const float inv = (range != 0.0f) ? __fdiv_rn(kNvfp4Range, range) : 0.0f;
+    uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * (a.K >> 1));
+
+    auto emit = [&](int kb, const uint4& x0, const uint4& x1) {
+        float v[16];
+        scale16(x0, x1, dv + 4 * kb, g, v);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(v[i], inv);
+        uint32_t lo, hi;
+        const uint32_t sb = nvfp4_encode_block(v, lo, hi);
+        crow[kb] = make_uint2(lo, hi);
+        if (sf_tiled) sf[nvfp4_sf_offset(row, kb, k64)] = static_cast<uint8_t>(sb);
+        else          sf[static_cast<size_t>(row) * n_blocks + kb] = static_cast<uint8_t>(sb);
+    };
+    if (NIT > 0) {
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
+            const int kb = it * 32 + lane;
+            if (kb < n_blocks) emit(kb, xr[2 * it], xr[2 * it + 1]);
+        }
+    } else {
+        for (int it = 0; it < n_it; ++it) {
+            const int kb = it * 32 + lane;
+            if (kb < n_blocks) emit(kb, ld_nc_16(xrow + 2 * kb), ld_nc_16(xrow + 2 * kb + 1));
+        }
+    }
+    if (lane == 0)
+        r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, kNvfp4Range), g) : 0.0f;
+}
+
+cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st)
+{
+    const int M_pad = sf_tiled ? ((a.M + 127) / 128) * 128 : a.M;
+    const int threads = 256;
+    const int blocks = (M_pad * 32 + threads - 1) / threads;
+    const int n_it = (a.K / 16 + 31) / 32;
+    const int tiled = sf_tiled ? 1 : 0;
+    if (n_it <= 2)       actq_nvfp4_kernel<2><<<blocks, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
+    else if (n_it <= 4)  actq_nvfp4_kernel<4><<<blocks, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
+    else if (n_it <= 8)  actq_nvfp4_kernel<8><<<blocks, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
+    else if (n_it <= 16) actq_nvfp4_kernel<16><<<blocks, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
+    else                 actq_nvfp4_kernel<0><<<blocks, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st)

@@ -53,7 +53,7 @@ rudder_status ensure_init()
     if (cudaGetDevice(&dev) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (dev < 0 || dev >= 64) return RUDDER_ERR_CUDA;
     if (!g_gemm_ready[dev]) {
-        if (gemm_i8_init() != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (gemm_i8_init() != cudaSuccess || gemm_fp4_init() != cudaSuccess) return RUDDER_ERR_CUDA;
         g_gemm_ready[dev] = true;
     }
     return RUDDER_OK;
@@ -87,8 +87,14 @@ int qmax_of(int scheme) { return scheme == RUDDER_W4A8_INT ? 127 : 7; }
 size_t workspace_bytes_for(const rudder_weight* w, int M)
 {
     if (!w || M < 1) return 0;
-    const size_t codes = align_up(static_cast<size_t>(M) * w->K, 256);
     const size_t r = align_up(static_cast<size_t>(M) * sizeof(float), 256);
+    if (w->scheme == RUDDER_W4A4_NVFP4) {
+        // packed E2M1 codes [M, K/2], block scales in tiled order for ceil(M/128) atoms, row scales
+        const size_t codes = align_up(static_cast<size_t>(M) * (w->K / 2), 256);
+        const size_t sf = align_up(static_cast<size_t>((M + 127) / 128) * (w->K / 64) * 512, 256);
+        return codes + sf + r;
+    }
+    const size_t codes = align_up(static_cast<size_t>(M) * w->K, 256);
     return codes + r;
 }
 
@@ -104,7 +110,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     if (s != RUDDER_OK) return s;
     if (!aligned(X, 16) || !aligned(Y, 16) || ldx % 8 != 0 || ldy % 8 != 0 || ldx < w->K || ldy < w->N) return RUDDER_ERR_ALIGN;
     if (bias && !aligned(bias, 16)) return RUDDER_ERR_ALIGN;
-    if (w->scheme != RUDDER_W4A8_INT && w->scheme != RUDDER_W4A4_INT) return RUDDER_ERR_UNSUPPORTED;
+    if (w->scheme == RUDDER_W4A4_NVFP4 && acc) return RUDDER_ERR_UNSUPPORTED;   // fp32 accumulation: nothing exact to dump
     const size_t need = workspace_bytes_for(w, M);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < need) return RUDDER_ERR_WORKSPACE;
     if (acc) {
@@ -113,14 +119,41 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     s = ensure_init();
     if (s != RUDDER_OK) return s;
 
-    int8_t* codes = static_cast<int8_t*>(workspace);
-    float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
-
     ActqArgs a;
     a.X = X; a.ldx = ldx; a.M = M; a.K = w->K; a.dinv = w->dinv;
     a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
     a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;
     a.seg = sp;
+
+    if (w->scheme == RUDDER_W4A4_NVFP4) {
+        uint8_t* ws = static_cast<uint8_t*>(workspace);
+        uint8_t* codes4 = ws;
+        uint8_t* sfx = ws + align_up(static_cast<size_t>(M) * (w->K / 2), 256);
+        float* r4 = reinterpret_cast<float*>(sfx + align_up(static_cast<size_t>((M + 127) / 128) * (w->K / 64) * 512, 256));
+        if (launch_actq_nvfp4(a, codes4, sfx, true, r4, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        GemmFp4Args g;
+        const int tt = gemm_fp4_token_tile(M);
+        const uint32_t box_tok = static_cast<uint32_t>(M < tt ? M : tt);
+        const uint64_t kb = static_cast<uint64_t>(w->K / 2);
+        if (!make_tmap_2d(&g.tm_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes4, kb, static_cast<uint64_t>(M), kb, 128, box_tok,
+                          CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap_2d(&g.tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w->codes, kb, static_cast<uint64_t>(w->N), kb, 128,
+                          static_cast<uint32_t>(w->N < 128 ? w->N : 128), CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !make_tmap_2d(&g.tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, static_cast<uint64_t>(w->N), static_cast<uint64_t>(M),
+                          static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128), box_tok,
+                          CU_TENSOR_MAP_SWIZZLE_NONE))
+            return RUDDER_ERR_CUDA;
+        g.sf_x = sfx; g.sf_w = w->sf_tiled;
+        g.M = M; g.N = w->N; g.K = w->K;
+        g.row_scale = r4; g.tensor_scale = w->tensor_scale; g.bias = bias;
+        if (launch_gemm_fp4(g, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        return RUDDER_OK;
+    }
+
+    int8_t* codes = static_cast<int8_t*>(workspace);
+    float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
     if (launch_actq_int(a, qmax_of(w->scheme), codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
 
@@ -168,8 +201,13 @@ rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, 
     if (out) *out = nullptr;
     if (!W || !out) return RUDDER_ERR_ARG;
     if (N < 64 || N % 64 != 0 || K < 128 || K % 128 != 0) return RUDDER_ERR_SHAPE;
-    if (scheme != RUDDER_W4A8_INT && scheme != RUDDER_W4A4_INT) return RUDDER_ERR_UNSUPPORTED;
-    if (!(group == 64 || group == 128 || group == K)) return RUDDER_ERR_SHAPE;
+    if (scheme != RUDDER_W4A8_INT && scheme != RUDDER_W4A4_INT && scheme != RUDDER_W4A4_NVFP4) return RUDDER_ERR_UNSUPPORTED;
+    if (scheme == RUDDER_W4A4_NVFP4) {
+        if (K % 256 != 0) return RUDDER_ERR_SHAPE;        // the block-scaled GEMM moves 256 input channels per stage
+        group = 16;
+    } else if (!(group == 64 || group == 128 || group == K)) {
+        return RUDDER_ERR_SHAPE;
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     rudder_status s = ensure_init();
     if (s != RUDDER_OK) return s;
@@ -180,6 +218,28 @@ rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, 
     cudaGetDevice(&w->device);
     const size_t n_groups = static_cast<size_t>(K / group);
     const size_t code_bytes = static_cast<size_t>(N) * (K / 2);
+    if (scheme == RUDDER_W4A4_NVFP4) {
+        const size_t sf_bytes = static_cast<size_t>((N + 127) / 128) * (K / 64) * 512;
+        unsigned int* amax_bits = nullptr;
+        bool ok4 = cudaMalloc(&w->codes, code_bytes) == cudaSuccess &&
+                   cudaMalloc(&w->scales_c, n_groups * N) == cudaSuccess &&
+                   cudaMalloc(&w->sf_tiled, sf_bytes) == cudaSuccess &&
+                   cudaMalloc(&w->dinv, static_cast<size_t>(K) * sizeof(float)) == cudaSuccess &&
+                   cudaMalloc(&w->tensor_scale, sizeof(float)) == cudaSuccess &&
+                   cudaMalloc(&amax_bits, sizeof(unsigned int)) == cudaSuccess;
+        w->bytes = code_bytes + n_groups * N + sf_bytes + static_cast<size_t>(K) * sizeof(float) + sizeof(float);
+        if (ok4)
+            ok4 = launch_pack_nvfp4(W, d, N, K, w->codes, static_cast<uint8_t*>(w->scales_c), w->sf_tiled, sf_bytes, w->dinv,
+                                    w->tensor_scale, amax_bits, st) == cudaSuccess &&
+                  cudaStreamSynchronize(st) == cudaSuccess;
+        if (amax_bits) cudaFree(amax_bits);
+        if (!ok4) {
+            rudder_weight_free(w);
+            return RUDDER_ERR_CUDA;
+        }
+        *out = w;
+        return RUDDER_OK;
+    }
     int8_t* tmp = nullptr;
     bool ok = cudaMalloc(&w->codes, code_bytes) == cudaSuccess &&
               cudaMalloc(&w->scales_t, n_groups * N * sizeof(float)) == cudaSuccess &&
@@ -232,10 +292,17 @@ rudder_status rudder_weight_export(const rudder_weight* w, uint8_t* codes, void*
 {
     if (!w) return RUDDER_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (codes && launch_export_int4(w->codes, w->N, w->K, codes, st) != cudaSuccess) return RUDDER_ERR_CUDA;
     const size_t n_groups = static_cast<size_t>(w->K / w->G);
-    if (scales && cudaMemcpyAsync(scales, w->scales_c, n_groups * w->N * sizeof(uint16_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-        return RUDDER_ERR_CUDA;
+    if (w->scheme == RUDDER_W4A4_NVFP4) {
+        if (codes && cudaMemcpyAsync(codes, w->codes, static_cast<size_t>(w->N) * (w->K / 2), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return RUDDER_ERR_CUDA;
+        if (scales && cudaMemcpyAsync(scales, w->scales_c, n_groups * w->N, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return RUDDER_ERR_CUDA;
+    } else {
+        if (codes && launch_export_int4(w->codes, w->N, w->K, codes, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (scales && cudaMemcpyAsync(scales, w->scales_c, n_groups * w->N * sizeof(uint16_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return RUDDER_ERR_CUDA;
+    }
     if (dinv && cudaMemcpyAsync(dinv, w->dinv, static_cast<size_t>(w->K) * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     if (tensor_scale && cudaMemcpyAsync(tensor_scale, w->tensor_scale, sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
@@ -390,19 +457,24 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
                                           const rudder_segments* seg, int step, const rudder_scale_table* tab,
                                           void* codes, uint8_t* block_scales, float* row_scale, void* stream)
 {
-    (void)block_scales;
     if (!w || !X || !codes || !row_scale) return RUDDER_ERR_ARG;
+    if (w->scheme == RUDDER_W4A4_NVFP4 && !block_scales) return RUDDER_ERR_ARG;
     if (M < 1) return RUDDER_ERR_SHAPE;
     SegParams sp;
     rudder_status s = check_table_and_segments(seg, step, tab, M, &sp);
     if (s != RUDDER_OK) return s;
     if (!aligned(X, 16) || ldx % 8 != 0 || ldx < w->K || !aligned(codes, 16)) return RUDDER_ERR_ALIGN;
-    if (w->scheme != RUDDER_W4A8_INT && w->scheme != RUDDER_W4A4_INT) return RUDDER_ERR_UNSUPPORTED;
     ActqArgs a;
     a.X = X; a.ldx = ldx; a.M = M; a.K = w->K; a.dinv = w->dinv;
     a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
     a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;
     a.seg = sp;
+    if (w->scheme == RUDDER_W4A4_NVFP4) {
+        // same kernel as production; the block scales go out row-major instead of in the tiled order
+        if (launch_actq_nvfp4(a, static_cast<uint8_t*>(codes), block_scales, false, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return RUDDER_ERR_CUDA;
+        return RUDDER_OK;
+    }
     if (launch_actq_int(a, qmax_of(w->scheme), static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     return RUDDER_OK;

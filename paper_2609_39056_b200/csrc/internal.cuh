@@ -64,6 +64,25 @@ cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G
 cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, cudaStream_t st);
 
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);
+cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st);
+cudaError_t launch_pack_nvfp4(const float* W, const float* d, int N, int K, uint8_t* codes, uint8_t* sb_canonical,
+                              uint8_t* sf_tiled, size_t sf_tiled_bytes, float* dinv, float* tensor_scale,
+                              unsigned int* amax_bits, cudaStream_t st);
+
+struct GemmFp4Args {
+    CUtensorMap tm_x;           // activation codes, packed E2M1 bytes [M, K/2], box {128 bytes, token tile}, 128-byte swizzle
+    CUtensorMap tm_w;           // weight codes, packed E2M1 bytes [N, K/2], box {128 bytes, 128 channels}, 128-byte swizzle
+    CUtensorMap tm_y;           // output bf16 [M, N]
+    const uint8_t* sf_x;        // activation block scales, tiled [ceil(M/128)][K/64][512]
+    const uint8_t* sf_w;        // weight block scales, tiled [ceil(N/128)][K/64][512]
+    int M, N, K;
+    const float* row_scale;     // r [M]
+    const float* tensor_scale;  // device [1]
+    const float* bias;
+};
+cudaError_t launch_gemm_fp4(const GemmFp4Args& a, cudaStream_t st);
+cudaError_t gemm_fp4_init();
+int gemm_fp4_token_tile(int M);
 
 struct GemmI8Args {
     CUtensorMap tm_x;           // activation codes int8 [M, K], box {128 bytes, token tile}, 128-byte swizzle

@@ -4,7 +4,9 @@
 #include "ptx.cuh"
 
 #include "pack.cu"
+#include "pack_nvfp4.cu"
 #include "actq.cu"
 #include "gemm_i8.cu"
+#include "gemm_fp4.cu"
 #include "api.cu"
 #include "static_ws.cu"
