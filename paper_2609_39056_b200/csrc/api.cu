@@ -47,6 +47,21 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 bool g_gemm_ready[64] = {false};
 
+int g_sm_count[64] = {0};
+
+int sm_count()
+{
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return 148;
+    if (g_sm_count[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        g_sm_count[dev] = n;
+    }
+    return g_sm_count[dev];
+}
+
 rudder_status ensure_init()
 {
     int dev = 0;
@@ -141,9 +156,10 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
             !make_tmap_2d(&g.tm_w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w->codes, kb, static_cast<uint64_t>(w->N), kb, 128,
                           static_cast<uint32_t>(w->N < 128 ? w->N : 128), CU_TENSOR_MAP_SWIZZLE_128B) ||
             !make_tmap_2d(&g.tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, static_cast<uint64_t>(w->N), static_cast<uint64_t>(M),
-                          static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128), box_tok,
-                          CU_TENSOR_MAP_SWIZZLE_NONE))
+                          static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128),
+                          static_cast<uint32_t>(M < gemm_fp4_store_rows(M) ? M : gemm_fp4_store_rows(M)), CU_TENSOR_MAP_SWIZZLE_NONE))
             return RUDDER_ERR_CUDA;
+        g.sm_count = sm_count();
         g.sf_x = sfx; g.sf_w = w->sf_tiled;
         g.M = M; g.N = w->N; g.K = w->K;
         g.row_scale = r4; g.tensor_scale = w->tensor_scale; g.bias = bias;

@@ -9,7 +9,10 @@
 //                of both sides (plain bulk copies of 512-byte chunks laid out in the tensor core's order)
 //   warp 1       allocates TMEM; converged loop, one elected lane copies the scales smem -> TMEM
 //                (tcgen05.cp) and issues the MMAs
-//   warps 4-11   epilogue: TMEM -> registers -> * (r_i s_W) + b_j -> bf16 -> shared -> TMA store
+//   warps 4-11   epilogue: TMEM -> registers (then TMEM is handed back at once) -> * (r_i s_W) + b_j
+//                -> bf16 -> shared, in two slabs per phase -> TMA stores
+// Persistent: one CTA per SM walks its tiles, so the epilogue of a tile overlaps the main loop of the
+// next one and TMEM / barriers are set up once.
 // TMEM: TT columns of fp32 accumulators, then two alternating regions of scale columns (4 columns per
 // 128 rows per MMA).
 #include "internal.cuh"
@@ -29,22 +32,24 @@ constexpr int NUM_THREADS = 384;
 constexpr int EPI_THREADS = 256;
 
 template <int TT> struct Tile {
-    static constexpr int S = (TT == 256) ? 4 : 6;                 // pipeline stages
+    static constexpr int S = (TT == 256) ? 3 : 5;                 // pipeline stages
     static constexpr int ATOMS = TT / 128;                        // 128-token scale atoms per tile
     static constexpr int X_BYTES = TT * KSTAGE_BYTES;
     static constexpr int W_BYTES = BN * KSTAGE_BYTES;
     static constexpr int SFW_BYTES = KSTEPS * SF_CHUNK;
     static constexpr int SFX_BYTES = ATOMS * KSTEPS * SF_CHUNK;
+    static constexpr int EC = TT / 2;                             // tokens per epilogue thread
+    static constexpr int SLAB_TOK = EC / 2;                       // tokens per staged slab (= TMA store box rows)
+    static constexpr int SLAB_BYTES = SLAB_TOK * BN * 2;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + S * X_BYTES;
     static constexpr int OFF_SFW = OFF_W + S * W_BYTES;
     static constexpr int OFF_SFX = OFF_SFW + S * SFW_BYTES;
-    static constexpr int BYTES = OFF_SFX + S * SFX_BYTES;
+    static constexpr int OFF_OUT = OFF_SFX + S * SFX_BYTES;       // two slabs of the bf16 output tile
+    static constexpr int BYTES = OFF_OUT + 2 * SLAB_BYTES;
     static constexpr int DYN_SMEM = BYTES + 1024;
     static constexpr int SF_COLS = KSTEPS * 4 * (1 + ATOMS);      // scale columns per region
     static constexpr int TMEM_COLS = (TT + 2 * SF_COLS > 256) ? 512 : 256;
-    static constexpr int EC = TT / 2;                             // tokens per epilogue thread
-    static_assert(S * X_BYTES >= TT * BN * 2, "the output tile is staged over the X ring");
 };
 
 struct Params {
@@ -57,9 +62,10 @@ struct Params {
     uint32_t x_tx, w_tx;
     int out_pitch;
     int m_atoms;                 // 128-row scale atoms that exist on the activation side
+    int m_tiles, n_tiles;        // token tiles, channel tiles
 };
 
-enum Where { W_EMPTY = 601, W_FULL = 701, W_ACC_FULL = 801 };
+enum Where { W_EMPTY = 601, W_FULL = 701, W_ACC_EMPTY = 702, W_ACC_FULL = 801 };
 
 __device__ __forceinline__ void sts16(uint32_t addr, uint16_t v) {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
@@ -103,6 +109,8 @@ __device__ __forceinline__ void umma_nvfp4(uint32_t tmem_d, uint64_t desc_a, uin
         : "memory");
 }
 
+// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...; consecutive tile indices walk the
+// token tiles of one channel tile, so CTAs running side by side share the same weight tile in L2.
 template <int TT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
@@ -110,27 +118,28 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 {
     using T = Tile<TT>;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * T::S + 1];
+    __shared__ __align__(8) uint64_t bars[2 * T::S + 2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_word;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * TT;
-    const int n0 = blockIdx.y * BN;
     const int n_stages = p.K / 256;
     const int k64 = p.K / 64;
+    const int total_tiles = p.m_tiles * p.n_tiles;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int i) { return bar0 + 8u * i; };
     auto empty = [&](int i) { return bar0 + 8u * (T::S + i); };
     const uint32_t acc_full = bar0 + 8u * (2 * T::S);
+    const uint32_t acc_empty = bar0 + 8u * (2 * T::S + 1);
 
     if (threadIdx.x == 0) {
         abort_word = 0;
         for (int i = 0; i < T::S; ++i) { mbar_init(full(i), 1); mbar_init(empty(i), 1); }
         mbar_init(acc_full, 1);
+        mbar_init(acc_empty, EPI_THREADS / 32);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -149,28 +158,32 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             tma_prefetch_desc(&tm_x);
             tma_prefetch_desc(&tm_w);
             tma_prefetch_desc(&tm_y);
-            // scale atoms of this tile that exist (the last token tile may own fewer)
-            int atoms = p.m_atoms - (m0 >> 7);
-            atoms = atoms > T::ATOMS ? T::ATOMS : atoms;
-            const uint32_t tx = p.x_tx + p.w_tx + T::SFW_BYTES + static_cast<uint32_t>(atoms) * KSTEPS * SF_CHUNK;
-            const uint8_t* sfw_src = p.sf_w + static_cast<size_t>(n0 >> 7) * k64 * SF_CHUNK;
             int issued = 0, slot = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int s = 0; s < n_stages; ++s) {
-                ok = mbar_wait<32>(empty(slot), ph ^ 1u, abortp, W_EMPTY);
-                if (!ok) break;
-                mbar_expect_tx(full(slot), tx);
-                tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, s * KSTAGE_BYTES, m0, full(slot));
-                tma_load_2d(smem_base + T::OFF_W + slot * T::W_BYTES, &tm_w, s * KSTAGE_BYTES, n0, full(slot));
-                bulk_load(smem_base + T::OFF_SFW + slot * T::SFW_BYTES, sfw_src + static_cast<size_t>(s) * T::SFW_BYTES,
-                          T::SFW_BYTES, full(slot));
-                for (int a = 0; a < atoms; ++a)
-                    bulk_load(smem_base + T::OFF_SFX + slot * T::SFX_BYTES + a * KSTEPS * SF_CHUNK,
-                              p.sf_x + (static_cast<size_t>((m0 >> 7) + a) * k64 + static_cast<size_t>(s) * KSTEPS) * SF_CHUNK,
-                              KSTEPS * SF_CHUNK, full(slot));
-                ++issued;
-                if (++slot == T::S) { slot = 0; ph ^= 1u; }
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % p.m_tiles) * TT;
+                const int n0 = (tile / p.m_tiles) * BN;
+                // scale atoms of this tile that exist (the last token tile may own fewer)
+                int atoms = p.m_atoms - (m0 >> 7);
+                atoms = atoms > T::ATOMS ? T::ATOMS : atoms;
+                const uint32_t tx = p.x_tx + p.w_tx + T::SFW_BYTES + static_cast<uint32_t>(atoms) * KSTEPS * SF_CHUNK;
+                const uint8_t* sfw_src = p.sf_w + static_cast<size_t>(n0 >> 7) * k64 * SF_CHUNK;
+                for (int s = 0; s < n_stages; ++s) {
+                    ok = mbar_wait<32>(empty(slot), ph ^ 1u, abortp, W_EMPTY);
+                    if (!ok) break;
+                    mbar_expect_tx(full(slot), tx);
+                    tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, s * KSTAGE_BYTES, m0, full(slot));
+                    tma_load_2d(smem_base + T::OFF_W + slot * T::W_BYTES, &tm_w, s * KSTAGE_BYTES, n0, full(slot));
+                    bulk_load(smem_base + T::OFF_SFW + slot * T::SFW_BYTES, sfw_src + static_cast<size_t>(s) * T::SFW_BYTES,
+                              T::SFW_BYTES, full(slot));
+                    for (int a = 0; a < atoms; ++a)
+                        bulk_load(smem_base + T::OFF_SFX + slot * T::SFX_BYTES + a * KSTEPS * SF_CHUNK,
+                                  p.sf_x + (static_cast<size_t>((m0 >> 7) + a) * k64 + static_cast<size_t>(s) * KSTEPS) * SF_CHUNK,
+                                  KSTEPS * SF_CHUNK, full(slot));
+                    ++issued;
+                    if (++slot == T::S) { slot = 0; ph ^= 1u; }
+                }
             }
             if (!ok) {
                 for (int i = max(0, issued - T::S); i < issued; ++i)
@@ -183,58 +196,81 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const uint32_t idesc = idesc_nvfp4(BN, TT);
         bool ok = true;
         int slot = 0;
-        uint32_t ph = 0;
-        for (int s = 0; s < n_stages; ++s) {
-            ok = mbar_wait(full(slot), ph, abortp, W_FULL);
+        uint32_t ph = 0, region = 0, tile_ph = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            // the accumulator is free once the epilogue has pulled the previous tile into registers
+            ok = mbar_wait(acc_empty, tile_ph ^ 1u, abortp, W_ACC_EMPTY);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tcgen05_fence_after_sync();
-            if (leader) {
-                const uint32_t sf_cols = tmem_base + TT + (s & 1) * T::SF_COLS;
-                const uint32_t sfw_smem = smem_base + T::OFF_SFW + slot * T::SFW_BYTES;
-                const uint32_t sfx_smem = smem_base + T::OFF_SFX + slot * T::SFX_BYTES;
-                const uint64_t da = umma_desc_sw128(smem_base + T::OFF_W + slot * T::W_BYTES);
-                const uint64_t db = umma_desc_sw128(smem_base + T::OFF_X + slot * T::X_BYTES);
+            for (int s = 0; s < n_stages; ++s) {
+                ok = mbar_wait(full(slot), ph, abortp, W_FULL);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tcgen05_fence_after_sync();
+                if (leader) {
+                    const uint32_t sf_cols = tmem_base + TT + region * T::SF_COLS;
+                    const uint32_t sfw_smem = smem_base + T::OFF_SFW + slot * T::SFW_BYTES;
+                    const uint32_t sfx_smem = smem_base + T::OFF_SFX + slot * T::SFX_BYTES;
+                    const uint64_t da = umma_desc_sw128(smem_base + T::OFF_W + slot * T::W_BYTES);
+                    const uint64_t db = umma_desc_sw128(smem_base + T::OFF_X + slot * T::X_BYTES);
 #pragma unroll
-                for (int j = 0; j < KSTEPS; ++j) {
-                    const uint32_t t_sfw = sf_cols + j * 4;
-                    const uint32_t t_sfx = sf_cols + KSTEPS * 4 + j * 4 * T::ATOMS;
-                    tmem_cp_sf(t_sfw, sf_desc(sfw_smem + j * SF_CHUNK));
+                    for (int j = 0; j < KSTEPS; ++j) {
+                        const uint32_t t_sfw = sf_cols + j * 4;
+                        const uint32_t t_sfx = sf_cols + KSTEPS * 4 + j * 4 * T::ATOMS;
+                        tmem_cp_sf(t_sfw, sf_desc(sfw_smem + j * SF_CHUNK));
 #pragma unroll
-                    for (int a = 0; a < T::ATOMS; ++a)
-                        tmem_cp_sf(t_sfx + a * 4, sf_desc(sfx_smem + (a * KSTEPS + j) * SF_CHUNK));
-                    umma_nvfp4(tmem_base, da + 2u * j, db + 2u * j, idesc, t_sfw, t_sfx, (s > 0 || j > 0) ? 1u : 0u);
+                        for (int a = 0; a < T::ATOMS; ++a)
+                            tmem_cp_sf(t_sfx + a * 4, sf_desc(sfx_smem + (a * KSTEPS + j) * SF_CHUNK));
+                        umma_nvfp4(tmem_base, da + 2u * j, db + 2u * j, idesc, t_sfw, t_sfx, (s > 0 || j > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty(slot));
+                    if (s == n_stages - 1) umma_commit(acc_full);
                 }
-                umma_commit(empty(slot));
-                if (s == n_stages - 1) umma_commit(acc_full);
+                __syncwarp();
+                region ^= 1u;
+                if (++slot == T::S) { slot = 0; ph ^= 1u; }
             }
-            __syncwarp();
-            if (++slot == T::S) { slot = 0; ph ^= 1u; }
+            tile_ph ^= 1u;
         }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ epilogue
         constexpr int EC = T::EC;
+        constexpr int SLAB = T::SLAB_TOK;
         const int q = warp & 3;
         const int h = (warp - 4) >> 2;
         const int ch_local = q * 32 + lane;
-        const int n = n0 + ch_local;
-        const bool n_ok = n < p.N;
-        const float b = (p.bias != nullptr && n_ok) ? __ldg(p.bias + n) : 0.0f;
         const float sw = __ldg(p.tensor_scale);
-        bool ok = mbar_wait<64>(acc_full, 0, abortp, W_ACC_FULL);
-        ok = __all_sync(0xffffffffu, ok);
-        if (ok) {
+        const uint32_t out0 = smem_base + T::OFF_OUT + h * T::SLAB_BYTES;    // this thread's slab
+        bool ok = true;
+        uint32_t tile_ph = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int m0 = (tile % p.m_tiles) * TT;
+            const int n0 = (tile / p.m_tiles) * BN;
+            const int n = n0 + ch_local;
+            const bool n_ok = n < p.N;
+            const float b = (p.bias != nullptr && n_ok) ? __ldg(p.bias + n) : 0.0f;
+            ok = mbar_wait<64>(acc_full, tile_ph, abortp, W_ACC_FULL);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tile_ph ^= 1u;
             tcgen05_fence_after_sync();
+            // Pull the thread's whole share of the accumulator into registers, then hand TMEM back: the
+            // next tile's MMAs run while this tile is scaled, converted and stored.
+            uint32_t v[EC];
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + h * EC;
-            const uint32_t stage0 = smem_base + T::OFF_X;       // every MMA has completed: the X ring is free
-#pragma unroll 1
-            for (int c = 0; c < EC / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32b_x32(taddr + c * 32, v);
-                tmem_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; j += 4) {
-                    const int tok = h * EC + c * 32 + j;
+            for (int c = 0; c < EC / 32; ++c) tmem_ld_32x32b_x32(taddr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&v[c * 32]));
+            tmem_wait_ld();
+            tcgen05_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty);
+#pragma unroll
+            for (int phase = 0; phase < 2; ++phase) {
+                // tokens [h EC + phase SLAB, + SLAB) of the tile go to slab h
+#pragma unroll
+                for (int j = 0; j < SLAB; j += 4) {
+                    const int tok = h * EC + phase * SLAB + j;
                     float4 rs = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (m0 + tok + 3 < p.M) {
                         rs = __ldg(reinterpret_cast<const float4*>(p.row_scale + m0 + tok));
@@ -247,22 +283,30 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     if (ch_local < p.out_pitch) {
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
-                            const float acc = n_ok ? __uint_as_float(v[j + t]) : 0.0f;
+                            const float acc = n_ok ? __uint_as_float(v[phase * SLAB + j + t]) : 0.0f;
                             const __nv_bfloat16 y = __float2bfloat16_rn(fmaf(acc, rr[t], b));
-                            sts16(stage0 + static_cast<uint32_t>((tok + t) * p.out_pitch + ch_local) * 2u, __bfloat16_as_ushort(y));
+                            sts16(out0 + static_cast<uint32_t>((j + t) * p.out_pitch + ch_local) * 2u, __bfloat16_as_ushort(y));
                         }
                     }
                 }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+                if (threadIdx.x == 128) {
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int tok0 = m0 + hh * EC + phase * SLAB;
+                        if (tok0 < p.M)
+                            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                         ::"l"(reinterpret_cast<uint64_t>(&tm_y)), "r"(smem_base + T::OFF_OUT + hh * T::SLAB_BYTES),
+                                           "r"(n0), "r"(tok0) : "memory");
+                    }
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");     // slabs may be overwritten again
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
             }
-            fence_proxy_async_smem();
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
-        if (ok && threadIdx.x == 128) {
-            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                         ::"l"(reinterpret_cast<uint64_t>(&tm_y)), "r"(smem_base + T::OFF_X), "r"(n0), "r"(m0) : "memory");
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        }
+        (void)ok;
     }
 
     tcgen05_fence_before_sync();
@@ -288,12 +332,16 @@ static cudaError_t launch_fp4_one(const GemmFp4Args& a, cudaStream_t st)
     p.w_tx = static_cast<uint32_t>(min(fp4::BN, a.N)) * fp4::KSTAGE_BYTES;
     p.out_pitch = min(fp4::BN, a.N);
     p.m_atoms = (a.M + 127) / 128;
-    dim3 grid((a.M + TT - 1) / TT, (a.N + fp4::BN - 1) / fp4::BN);
+    p.m_tiles = (a.M + TT - 1) / TT;
+    p.n_tiles = (a.N + fp4::BN - 1) / fp4::BN;
+    const int tiles = p.m_tiles * p.n_tiles;
+    const int grid = tiles < a.sm_count ? tiles : a.sm_count;
     fp4::gemm_nvfp4_kernel<TT><<<grid, fp4::NUM_THREADS, T::DYN_SMEM, st>>>(a.tm_x, a.tm_w, a.tm_y, p);
     return cudaGetLastError();
 }
 
 int gemm_fp4_token_tile(int M) { return M > 128 ? 256 : 128; }
+int gemm_fp4_store_rows(int M) { return gemm_fp4_token_tile(M) / 4; }
 
 cudaError_t gemm_fp4_init()
 {

@@ -79,7 +79,9 @@ struct GemmFp4Args {
     const float* row_scale;     // r [M]
     const float* tensor_scale;  // device [1]
     const float* bias;
+    int sm_count;               // persistent grid size
 };
+int gemm_fp4_store_rows(int M); // token rows of one TMA store box (a quarter of the token tile)
 cudaError_t launch_gemm_fp4(const GemmFp4Args& a, cudaStream_t st);
 cudaError_t gemm_fp4_init();
 int gemm_fp4_token_tile(int M);
