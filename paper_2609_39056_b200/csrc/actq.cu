@@ -129,35 +129,34 @@ __global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int
         r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, static_cast<float>(qmax)), g) : 0.0f;
 }
 
-// ---- rows spread over TPR threads ---------------------------------------------------------------
-// The warp-per-row kernels above keep a whole row in one warp's registers, which caps the occupancy
-// (171 registers at K = 8192) and leaves the memory system idle while a warp computes.  Here a row is
-// spread over TPR threads of a 256-thread CTA (256 / TPR rows per CTA), each thread holding at most
-// NCH 16-byte pieces, so that registers stay low and many rows are in flight per SM.
-// Range pass: max_k |x dinv| and one multiplication by gamma -- identical bits to max_k |(x dinv) gamma|
-// because rounding is monotonic and gamma > 0.
-template <int TPR>
-__device__ __forceinline__ float row_max(float m, float* red /* [8] shared */, int row_in_cta, int tid_in_row) {
+// ---- one row per CTA step ------------------------------------------------------------------------
+// The warp-per-row kernels above keep a whole row in one warp's registers, which caps the occupancy and
+// leaves the memory system idle while a warp computes.  Here a row is spread over the T threads of a
+// CTA (T = row pieces, up to 1024; NCH pieces per thread for longer rows).  The CTA is persistent: it
+// walks rows blockIdx.x, blockIdx.x + gridDim.x, ..., so a thread always meets the same input channels
+// and keeps their dinv in registers, and it issues the loads of its next row before working on the
+// current one.  Range pass: max_k |x dinv| and one multiplication by gamma -- identical bits to
+// max_k |(x dinv) gamma| because rounding is monotonic and gamma > 0.
+__device__ __forceinline__ float block_max(float m, float* red /* [32] shared */) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (TPR == 32) return m;
-    constexpr int WPR = TPR / 32;                  // warps per row
-    const int w_in_row = tid_in_row >> 5;
-    if ((tid_in_row & 31) == 0) red[row_in_cta * WPR + w_in_row] = m;
+    const int n_warps = (blockDim.x + 31) >> 5;
+    if (n_warps == 1) return m;
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
     __syncthreads();
-    float r = red[row_in_cta * WPR];
+    float r = (static_cast<int>(threadIdx.x & 31) < n_warps) ? red[threadIdx.x & 31] : 0.0f;
 #pragma unroll
-    for (int i = 1; i < WPR; ++i) r = fmaxf(r, red[row_in_cta * WPR + i]);
+    for (int o = 16; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, o));
     return r;
 }
 
-__device__ __forceinline__ void absmax8(const uint4& x, const float4& d0, const float4& d1, float& m) {
+// x (8 bf16) * dinv -> 8 fp32 (the first of the two roundings of v = (x dinv) gamma)
+__device__ __forceinline__ void mul_dinv8(const uint4& x, const float (&dd)[8], float (&u)[8]) {
     const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-    const float dd[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        m = fmaxf(m, fabsf(__fmul_rn(__uint_as_float(w[i] << 16), dd[2 * i])));
-        m = fmaxf(m, fabsf(__fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), dd[2 * i + 1])));
+        u[2 * i] = __fmul_rn(__uint_as_float(w[i] << 16), dd[2 * i]);
+        u[2 * i + 1] = __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), dd[2 * i + 1]);
     }
 }
 
@@ -180,55 +179,67 @@ __device__ __forceinline__ uint2 round8_fast(const float (&v)[8], float inv, flo
     return make_uint2(lo, hi);
 }
 
-template <int TPR, int NCH>
-__global__ void __launch_bounds__(256) actq_int_rows_kernel(ActqArgs a, int qmax, int8_t* __restrict__ codes, int64_t ldc,
+template <int NCH>
+__global__ void __launch_bounds__(1024) actq_int_row_kernel(ActqArgs a, int qmax, int8_t* __restrict__ codes, int64_t ldc,
                                                              float* __restrict__ r)
 {
-    __shared__ float red[8];
-    constexpr int RPC = 256 / TPR;                 // rows per CTA
-    const int row_in_cta = threadIdx.x / TPR;
-    const int t = threadIdx.x % TPR;
-    const int row = blockIdx.x * RPC + row_in_cta;
-    const bool live = row < a.M;                   // whole rows are live or not: no divergence inside a row
+    __shared__ float red[2][32];
+    const int t = threadIdx.x;
+    const int T = blockDim.x;
     const int n_chunks = a.K >> 3;
-    const float4* dv = reinterpret_cast<const float4*>(a.dinv);
-    const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(live ? row : 0) * a.ldx);
-    const float g = live ? a.gamma_step[stream_of_row(a.seg, row)] : 1.0f;
+    const float qmaxf = static_cast<float>(qmax);
 
-    uint4 xr[NCH];
+    float dd[NCH][8];
 #pragma unroll
     for (int i = 0; i < NCH; ++i) {
-        const int c = i * TPR + t;
-        xr[i] = (live && c < n_chunks) ? ld_nc_16(xrow + c) : make_uint4(0, 0, 0, 0);
+        const int c = i * T + t;
+        const float4 d0 = (c < n_chunks) ? __ldg(reinterpret_cast<const float4*>(a.dinv) + 2 * c) : make_float4(0, 0, 0, 0);
+        const float4 d1 = (c < n_chunks) ? __ldg(reinterpret_cast<const float4*>(a.dinv) + 2 * c + 1) : make_float4(0, 0, 0, 0);
+        dd[i][0] = d0.x; dd[i][1] = d0.y; dd[i][2] = d0.z; dd[i][3] = d0.w;
+        dd[i][4] = d1.x; dd[i][5] = d1.y; dd[i][6] = d1.z; dd[i][7] = d1.w;
     }
-    float range;
-    if (a.clip_step == nullptr) {
+    auto load_row = [&](int row, uint4 (&x)[NCH]) {
+        const bool live = row < a.M;
+        const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(live ? row : 0) * a.ldx);
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int c = i * T + t;
+            x[i] = (live && c < n_chunks) ? ld_nc_16(xrow + c) : make_uint4(0, 0, 0, 0);
+        }
+    };
+
+    uint4 nxt[NCH];
+    load_row(blockIdx.x, nxt);
+    int par = 0;
+    for (int row = blockIdx.x; row < a.M; row += gridDim.x, par ^= 1) {
+        float u[NCH][8];
         float m = 0.0f;
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
-            const int c = i * TPR + t;
-            if (c < n_chunks) absmax8(xr[i], __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), m);
-        }
-        range = __fmul_rn(row_max<TPR>(m, red, row_in_cta, t), g);
-    } else {
-        range = *a.clip_step;
-    }
-    if (!live) return;
-    const float inv = (range != 0.0f) ? __fdiv_rn(static_cast<float>(qmax), range) : 0.0f;
-    const float qmaxf = static_cast<float>(qmax);
-    uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldc);
+            mul_dinv8(nxt[i], dd[i], u[i]);       // pieces past the row end are zero
 #pragma unroll
-    for (int i = 0; i < NCH; ++i) {
-        const int c = i * TPR + t;
-        if (c < n_chunks) {
-            float v[8];
-            scale8(xr[i], __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
-            crow[c] = (a.clip_step == nullptr) ? round8_fast<false>(v, inv, qmaxf) : round8_fast<true>(v, inv, qmaxf);
+            for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(u[i][j]));
         }
+        load_row(row + gridDim.x, nxt);            // prefetch the next row
+        const float g = a.gamma_step[stream_of_row(a.seg, row)];
+        float range;
+        if (a.clip_step == nullptr) range = __fmul_rn(block_max(m, red[par]), g);
+        else                        range = *a.clip_step;
+        const float inv = (range != 0.0f) ? __fdiv_rn(qmaxf, range) : 0.0f;
+        uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldc);
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int c = i * T + t;
+            if (c < n_chunks) {
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[j] = __fmul_rn(u[i][j], g);
+                crow[c] = (a.clip_step == nullptr) ? round8_fast<false>(v, inv, qmaxf) : round8_fast<true>(v, inv, qmaxf);
+            }
+        }
+        if (t == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, qmaxf), g) : 0.0f;
     }
-    if (t == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, qmaxf), g) : 0.0f;
 }
-
 
 // ---- NVFP4 activations -------------------------------------------------------------------------
 // One warp per row; a lane owns one block of 16 channels per step (two 16-byte loads), so a warp step
@@ -327,109 +338,133 @@ __global__ void __launch_bounds__(256) actq_nvfp4_kernel(ActqArgs a, int M_pad, 
         r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, kNvfp4Range), g) : 0.0f;
 }
 
-template <int TPR, int NCH>
-__global__ void __launch_bounds__(256) actq_nvfp4_rows_kernel(ActqArgs a, int M_pad, uint8_t* __restrict__ codes,
+template <int NCH>
+__global__ void __launch_bounds__(1024) actq_nvfp4_row_kernel(ActqArgs a, int M_pad, uint8_t* __restrict__ codes,
                                                                uint8_t* __restrict__ sf, int sf_tiled, float* __restrict__ r)
 {
-    __shared__ float red[8];
-    constexpr int RPC = 256 / TPR;
-    const int row_in_cta = threadIdx.x / TPR;
-    const int t = threadIdx.x % TPR;
-    const int row = blockIdx.x * RPC + row_in_cta;
+    __shared__ float red[2][32];
+    const int t = threadIdx.x;
+    const int T = blockDim.x;
+    const int lane = t & 31;
     const int n_blocks = a.K >> 4;
     const int k64 = a.K >> 6;
-    const bool live = row < a.M;
-    if (!live && row < M_pad) {                    // padding row of the last 128-row scale atom
-        for (int kb = t; kb < n_blocks; kb += TPR) sf[nvfp4_sf_offset(row, kb, k64)] = 0;
-    }
-    const float4* dv = reinterpret_cast<const float4*>(a.dinv);
-    const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(live ? row : 0) * a.ldx);
-    const float g = live ? a.gamma_step[stream_of_row(a.seg, row)] : 1.0f;
 
-    uint4 xr[2 * NCH];
+    float dd[NCH][16];
 #pragma unroll
     for (int i = 0; i < NCH; ++i) {
-        const int kb = i * TPR + t;
-        const bool in = live && kb < n_blocks;
-        xr[2 * i] = in ? ld_nc_16(xrow + 2 * kb) : make_uint4(0, 0, 0, 0);
-        xr[2 * i + 1] = in ? ld_nc_16(xrow + 2 * kb + 1) : make_uint4(0, 0, 0, 0);
+        const int kb = i * T + t;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float4 d4 = (kb < n_blocks) ? __ldg(reinterpret_cast<const float4*>(a.dinv) + 4 * kb + j) : make_float4(0, 0, 0, 0);
+            dd[i][4 * j] = d4.x; dd[i][4 * j + 1] = d4.y; dd[i][4 * j + 2] = d4.z; dd[i][4 * j + 3] = d4.w;
+        }
     }
-    float range;
-    if (a.clip_step == nullptr) {
+    auto load_row = [&](int row, uint4 (&x)[2 * NCH]) {
+        const bool live = row < a.M;
+        const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(live ? row : 0) * a.ldx);
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) {
+            const int kb = i * T + t;
+            const bool in = live && kb < n_blocks;
+            x[2 * i] = in ? ld_nc_16(xrow + 2 * kb) : make_uint4(0, 0, 0, 0);
+            x[2 * i + 1] = in ? ld_nc_16(xrow + 2 * kb + 1) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    // four neighbouring lanes own the four blocks of one 64-channel step: one 32-bit store for their scales
+    auto store_sf = [&](int row, int kb, uint32_t sb) {
+        uint32_t word = sb << (8 * (lane & 3));
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        if ((lane & 3) == 0 && kb < n_blocks) {
+            const size_t off = sf_tiled ? nvfp4_sf_offset(row, kb, k64) : static_cast<size_t>(row) * n_blocks + kb;
+            *reinterpret_cast<uint32_t*>(sf + off) = word;
+        }
+    };
+
+    uint4 nxt[2 * NCH];
+    load_row(blockIdx.x, nxt);
+    int par = 0;
+    for (int row = blockIdx.x; row < M_pad; row += gridDim.x, par ^= 1) {
+        if (row >= a.M) {                          // padding row of the last 128-row scale atom: zero scales
+#pragma unroll
+            for (int i = 0; i < NCH; ++i) store_sf(row, i * T + t, 0u);
+            continue;
+        }
+        float u[NCH][16];
         float m = 0.0f;
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
-            const int kb = i * TPR + t;
-            if (kb < n_blocks) {
-                absmax8(xr[2 * i], __ldg(dv + 4 * kb), __ldg(dv + 4 * kb + 1), m);
-                absmax8(xr[2 * i + 1], __ldg(dv + 4 * kb + 2), __ldg(dv + 4 * kb + 3), m);
+            float lo8[8], hi8[8];
+            mul_dinv8(nxt[2 * i], *reinterpret_cast<const float(*)[8]>(&dd[i][0]), lo8);
+            mul_dinv8(nxt[2 * i + 1], *reinterpret_cast<const float(*)[8]>(&dd[i][8]), hi8);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                u[i][j] = lo8[j];
+                u[i][8 + j] = hi8[j];
+                m = fmaxf(m, fmaxf(fabsf(lo8[j]), fabsf(hi8[j])));
             }
         }
-        range = __fmul_rn(row_max<TPR>(m, red, row_in_cta, t), g);
-    } else {
-        range = *a.clip_step;
-    }
-    if (!live) return;
-    const float inv = (range != 0.0f) ? __fdiv_rn(kNvfp4Range, range) : 0.0f;
-    uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * (a.K >> 1));
+        load_row(row + gridDim.x, nxt);
+        const float g = a.gamma_step[stream_of_row(a.seg, row)];
+        float range;
+        if (a.clip_step == nullptr) range = __fmul_rn(block_max(m, red[par]), g);
+        else                        range = *a.clip_step;
+        const float inv = (range != 0.0f) ? __fdiv_rn(kNvfp4Range, range) : 0.0f;
+        uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * (a.K >> 1));
 #pragma unroll
-    for (int i = 0; i < NCH; ++i) {
-        const int kb = i * TPR + t;
-        if (kb < n_blocks) {
+        for (int i = 0; i < NCH; ++i) {
+            const int kb = i * T + t;
             float v[16];
-            scale16(xr[2 * i], xr[2 * i + 1], dv + 4 * kb, g, v);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(v[j], inv);
+            for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(__fmul_rn(u[i][j], g), inv);
             uint32_t lo, hi;
             const uint32_t sb = nvfp4_encode_block(v, lo, hi);
-            crow[kb] = make_uint2(lo, hi);
-            if (sf_tiled) sf[nvfp4_sf_offset(row, kb, k64)] = static_cast<uint8_t>(sb);
-            else          sf[static_cast<size_t>(row) * n_blocks + kb] = static_cast<uint8_t>(sb);
+            if (kb < n_blocks) crow[kb] = make_uint2(lo, hi);
+            store_sf(row, kb, sb);
         }
+        if (t == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, kNvfp4Range), g) : 0.0f;
     }
-    if (t == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, kNvfp4Range), g) : 0.0f;
+}
+
+// Threads per CTA and pieces per thread for a row of n pieces.
+static void row_launch_shape(int n, int& threads, int& nch) {
+    nch = (n + 1023) / 1024;
+    threads = ((n + nch - 1) / nch + 31) / 32 * 32;
+}
+static int row_grid(int rows, int threads) {
+    const int per_sm = 2048 / threads > 0 ? 2048 / threads : 1;
+    const int cap = 148 * (per_sm > 8 ? 8 : per_sm);
+    return rows < cap ? rows : cap;
 }
 
 cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st)
 {
     const int M_pad = sf_tiled ? ((a.M + 127) / 128) * 128 : a.M;
     const int tiled = sf_tiled ? 1 : 0;
-    const int n_blocks = a.K / 16;
-#define RUDDER_FP4_ROWS(TPR, NCH)                                                                                  \
-    actq_nvfp4_rows_kernel<TPR, NCH><<<(M_pad + 256 / TPR - 1) / (256 / TPR), 256, 0, st>>>(a, M_pad, codes, sf, tiled, r)
-    if (n_blocks <= 32)        RUDDER_FP4_ROWS(32, 1);
-    else if (n_blocks <= 64)   RUDDER_FP4_ROWS(64, 1);
-    else if (n_blocks <= 128)  RUDDER_FP4_ROWS(128, 1);
-    else if (n_blocks <= 256)  RUDDER_FP4_ROWS(256, 1);
-    else if (n_blocks <= 512)  RUDDER_FP4_ROWS(256, 2);
-    else if (n_blocks <= 768)  RUDDER_FP4_ROWS(256, 3);
-    else if (n_blocks <= 1024) RUDDER_FP4_ROWS(256, 4);
+    int threads, nch;
+    row_launch_shape(a.K / 16, threads, nch);
+    const int grid = row_grid(M_pad, threads);
+    if (nch == 1)      actq_nvfp4_row_kernel<1><<<grid, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
+    else if (nch == 2) actq_nvfp4_row_kernel<2><<<grid, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
     else {
         const int blocks = (M_pad * 32 + 255) / 256;      // very long rows: one warp per row, row read twice
         actq_nvfp4_kernel<0><<<blocks, 256, 0, st>>>(a, M_pad, codes, sf, tiled, r);
     }
-#undef RUDDER_FP4_ROWS
     return cudaGetLastError();
 }
 
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st)
 {
-    const int n_chunks = a.K / 8;
-#define RUDDER_INT_ROWS(TPR, NCH)                                                                                  \
-    actq_int_rows_kernel<TPR, NCH><<<(a.M + 256 / TPR - 1) / (256 / TPR), 256, 0, st>>>(a, qmax, codes, ldc, r)
-    if (n_chunks <= 32)        RUDDER_INT_ROWS(32, 1);
-    else if (n_chunks <= 64)   RUDDER_INT_ROWS(64, 1);
-    else if (n_chunks <= 128)  RUDDER_INT_ROWS(128, 1);
-    else if (n_chunks <= 256)  RUDDER_INT_ROWS(256, 1);
-    else if (n_chunks <= 512)  RUDDER_INT_ROWS(256, 2);
-    else if (n_chunks <= 1024) RUDDER_INT_ROWS(256, 4);
-    else if (n_chunks <= 1536) RUDDER_INT_ROWS(256, 6);
-    else if (n_chunks <= 2048) RUDDER_INT_ROWS(256, 8);
+    int threads, nch;
+    row_launch_shape(a.K / 8, threads, nch);
+    const int grid = row_grid(a.M, threads);
+    if (nch == 1)      actq_int_row_kernel<1><<<grid, threads, 0, st>>>(a, qmax, codes, ldc, r);
+    else if (nch == 2) actq_int_row_kernel<2><<<grid, threads, 0, st>>>(a, qmax, codes, ldc, r);
+    else if (nch <= 4) actq_int_row_kernel<4><<<grid, threads, 0, st>>>(a, qmax, codes, ldc, r);
     else {
         const int blocks = (a.M * 32 + 255) / 256;         // very long rows: one warp per row, row read twice
         actq_int_kernel<0><<<blocks, 256, 0, st>>>(a, qmax, codes, ldc, r);
     }
-#undef RUDDER_INT_ROWS
     return cudaGetLastError();
 }
 

@@ -116,7 +116,7 @@ enum Where {   // codes recorded when a bounded wait gives up
     W_X_EMPTY = 101,
     W_W_EMPTY = 201,
     W_X_FULL = 301, W_W_FULL = 302, W_ACC_EMPTY = 303,
-    W_ACC_FULL = 401
+    W_ACC_FULL = 401, W_RS_FULL = 402
 };
 
 __device__ __forceinline__ void sts128(uint32_t addr, const uint4& v) {
@@ -145,7 +145,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 {
     using T = Tile<TT>;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * SW + 4];
+    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * SW + 5];
+    __shared__ __align__(16) float rs_smem[TT];      // row scales r_i of the tile's tokens (0 past M)
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_word;
 
@@ -164,12 +165,14 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     auto w_empty = [&](int i) { return bar0 + 8u * (2 * T::SX + SW + i); };
     auto acc_full = [&](int i) { return bar0 + 8u * (2 * T::SX + 2 * SW + i); };
     auto acc_empty = [&](int i) { return bar0 + 8u * (2 * T::SX + 2 * SW + 2 + i); };
+    const uint32_t rs_full = bar0 + 8u * (2 * T::SX + 2 * SW + 4);
 
     if (threadIdx.x == 0) {
         abort_word = 0;
         for (int i = 0; i < T::SX; ++i) { mbar_init(x_full(i), 1); mbar_init(x_empty(i), 1); }
         for (int i = 0; i < SW; ++i) { mbar_init(w_full(i), UNPACK_THREADS / 32); mbar_init(w_empty(i), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(acc_full(i), 1); mbar_init(acc_empty(i), EPI_THREADS / 32); }
+        mbar_init(rs_full, 1);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -274,6 +277,11 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #endif
             if (leader) { PROF_PUT(3, x_full); PROF_PUT(4, w_full); PROF_PUT(5, acc_empty); PROF_PUT(6, mma_total); }
         }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ row scales of the tile -> shared
+        for (int i = lane; i < TT; i += 32) rs_smem[i] = (m0 + i < p.M) ? __ldg(p.row_scale + m0 + i) : 0.0f;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(rs_full);
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ INT4 -> int8 unpack
         // 128 channels x 64 packed bytes per stage = 512 16-byte pieces, 4 per thread: piece idx covers
@@ -371,11 +379,13 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             if (g + 2 < n_groups) sc_next2 = ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + 2) * p.N);
 #endif
 #ifndef RUDDER_DBG_EPI_FREE
-            ok = PROF_WAIT(acc_full, mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), (g >> 1) & 1, abortp, W_ACC_FULL));
+            // lane 0 polls, the others wait at the shuffle: no 32-way spin, and the verdict is warp-uniform
+            // (the TMEM loads below are warp-collective)
+            if (lane == 0) ok = PROF_WAIT(acc_full, mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), (g >> 1) & 1, abortp, W_ACC_FULL));
 #ifdef RUDDER_ROLE_PROF
             const long long v_t0 = clock64();
 #endif
-            ok = __all_sync(0xffffffffu, ok);     // warp-uniform: the TMEM loads below are warp-collective
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
 #endif
 #ifdef RUDDER_ROLE_PROF
@@ -448,27 +458,21 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #endif
         // The last acc_full arrives after every MMA of the tile has completed, so the X ring is free:
         // stage the transposed bf16 tile there ([token][channel], `out_pitch` channels per row).
+        if (ok) ok = mbar_wait<64>(rs_full, 0, abortp, W_RS_FULL);
         if (ok) {
             const float b = (p.bias != nullptr && n_ok) ? __ldg(p.bias + n) : 0.0f;
             const uint32_t stage0 = smem_base + T::OFF_X;
+            const float4* rs4 = reinterpret_cast<const float4*>(rs_smem + h * EC);
+            if (ch_local < p.out_pitch) {
+                uint32_t dst = stage0 + static_cast<uint32_t>(h * EC * p.out_pitch + ch_local) * 2u;
+                const uint32_t step = static_cast<uint32_t>(p.out_pitch) * 2u;
 #pragma unroll
-            for (int j = 0; j < EC; j += 4) {
-                const int tok = h * EC + j;                      // token within the tile
-                float4 rs = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (m0 + tok + 3 < p.M) {
-                    rs = __ldg(reinterpret_cast<const float4*>(p.row_scale + m0 + tok));   // (m0 + tok) % 4 == 0
-                } else {
-                    if (m0 + tok + 0 < p.M) rs.x = __ldg(p.row_scale + m0 + tok + 0);
-                    if (m0 + tok + 1 < p.M) rs.y = __ldg(p.row_scale + m0 + tok + 1);
-                    if (m0 + tok + 2 < p.M) rs.z = __ldg(p.row_scale + m0 + tok + 2);
-                }
-                const float rr[4] = {rs.x, rs.y, rs.z, rs.w};
-                if (ch_local < p.out_pitch) {
-#pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        const __nv_bfloat16 v = __float2bfloat16_rn(fmaf(acc[j + t], rr[t], b));
-                        sts16(stage0 + static_cast<uint32_t>((tok + t) * p.out_pitch + ch_local) * 2u, __bfloat16_as_ushort(v));
-                    }
+                for (int j = 0; j < EC; j += 4) {
+                    const float4 rs = rs4[j >> 2];                   // broadcast read, zero past M
+                    sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 0], rs.x, b)))); dst += step;
+                    sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 1], rs.y, b)))); dst += step;
+                    sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 2], rs.z, b)))); dst += step;
+                    sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 3], rs.w, b)))); dst += step;
                 }
             }
             fence_proxy_async_smem();                            // generic writes -> visible to the TMA store
