@@ -30,6 +30,7 @@ constexpr int KSTEPS = 4;          // MMAs (K = 64) per stage
 constexpr int SF_CHUNK = 512;      // scale bytes of 128 rows x 64 input channels
 constexpr int NUM_THREADS = 384;
 constexpr int EPI_THREADS = 256;
+constexpr int kGroupM = 16;        // token tiles per rasterisation group (their activation rows stay in L2)
 
 template <int TT> struct Tile {
     static constexpr int S = (TT == 256) ? 3 : 5;                 // pipeline stages
@@ -109,8 +110,7 @@ __device__ __forceinline__ void umma_nvfp4(uint32_t tmem_d, uint64_t desc_a, uin
         : "memory");
 }
 
-// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...; consecutive tile indices walk the
-// token tiles of one channel tile, so CTAs running side by side share the same weight tile in L2.
+// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ... in the grouped order of tile_coords.
 template <int TT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
@@ -162,8 +162,10 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             uint32_t ph = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.m_tiles) * TT;
-                const int n0 = (tile / p.m_tiles) * BN;
+                int tm, tn;
+                tile_coords(tile, p.m_tiles, p.n_tiles, kGroupM, tm, tn);
+                const int m0 = tm * TT;
+                const int n0 = tn * BN;
                 // scale atoms of this tile that exist (the last token tile may own fewer)
                 int atoms = p.m_atoms - (m0 >> 7);
                 atoms = atoms > T::ATOMS ? T::ATOMS : atoms;
@@ -245,8 +247,10 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         bool ok = true;
         uint32_t tile_ph = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-            const int m0 = (tile % p.m_tiles) * TT;
-            const int n0 = (tile / p.m_tiles) * BN;
+            int tm, tn;
+            tile_coords(tile, p.m_tiles, p.n_tiles, kGroupM, tm, tn);
+            const int m0 = tm * TT;
+            const int n0 = tn * BN;
             const int n = n0 + ch_local;
             const bool n_ok = n < p.N;
             const float b = (p.bias != nullptr && n_ok) ? __ldg(p.bias + n) : 0.0f;

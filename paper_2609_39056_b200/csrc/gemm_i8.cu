@@ -95,6 +95,7 @@ struct Params {
     const float* bias;           // [N] or nullptr
     int32_t* acc;                // accumulator dump [K/G][rows][cols] or nullptr
     int row0, rows, col0, cols;
+    int m_tiles, n_tiles;        // token tiles, channel tiles (grid = m_tiles * n_tiles CTAs)
     uint32_t x_tx;               // bytes one activation TMA box delivers
     int out_pitch;               // channels per row of the staged output tile (= TMA store box width)
 #ifdef RUDDER_ROLE_PROF
@@ -105,7 +106,7 @@ struct Params {
 #ifdef RUDDER_ROLE_PROF
 #define PROF_DECL(n) long long prof_##n = 0
 #define PROF_WAIT(n, expr) [&]() { const long long t_ = clock64(); const bool r_ = (expr); prof_##n += clock64() - t_; return r_; }()
-#define PROF_PUT(i, n) do { if (blockIdx.x == 0 && blockIdx.y == 0 && p.prof) p.prof[i] = prof_##n; } while (0)
+#define PROF_PUT(i, n) do { if (blockIdx.x == 0 && p.prof) p.prof[i] = prof_##n; } while (0)
 #else
 #define PROF_DECL(n)
 #define PROF_WAIT(n, expr) (expr)
@@ -152,8 +153,10 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * TT;          // first token of the tile
-    const int n0 = blockIdx.y * BN;          // first output channel of the tile
+    int tile_m, tile_n;
+    tile_coords(blockIdx.x, p.m_tiles, p.n_tiles, 16, tile_m, tile_n);
+    const int m0 = tile_m * TT;              // first token of the tile
+    const int n0 = tile_n * BN;              // first output channel of the tile
     const int n_stages = p.K / KSTAGE;
     const int n_groups = p.K / p.G;
 
@@ -517,8 +520,9 @@ static cudaError_t launch_one(const GemmI8Args& a, cudaStream_t st)
     p.prof = reinterpret_cast<long long*>(a.acc);   // development build only: the dump pointer carries the counters
     p.acc = nullptr;
 #endif
-    dim3 grid((a.M + TT - 1) / TT, (a.N + BN - 1) / BN);
-    gemm_i8_w4_kernel<TT, DUMP><<<grid, NUM_THREADS, T::DYN_SMEM, st>>>(a.tm_x, a.tm_y, p);
+    p.m_tiles = (a.M + TT - 1) / TT;
+    p.n_tiles = (a.N + BN - 1) / BN;
+    gemm_i8_w4_kernel<TT, DUMP><<<p.m_tiles * p.n_tiles, NUM_THREADS, T::DYN_SMEM, st>>>(a.tm_x, a.tm_y, p);
     return cudaGetLastError();
 }
 

@@ -88,6 +88,20 @@ __device__ __forceinline__ bool elect_one() {
     return is_leader != 0;
 }
 
+// ---- tile rasterisation --------------------------------------------------------------------------
+// Tile t -> (token tile m, channel tile n): token tiles are taken in groups of `gm`; inside a group
+// the order is n-major, m fastest.  CTAs that run side by side then share one slab of activation rows
+// (gm token tiles, small enough to stay in L2) across all channel tiles, instead of streaming the
+// whole activation matrix from DRAM once per wave.
+__device__ __forceinline__ void tile_coords(int t, int m_tiles, int n_tiles, int gm, int& m, int& n) {
+    const int per_group = gm * n_tiles;
+    const int grp = t / per_group;
+    const int rem = t - grp * per_group;
+    const int m_in = min(gm, m_tiles - grp * gm);
+    n = rem / m_in;
+    m = grp * gm + (rem - n * m_in);
+}
+
 // ---- proxies / fences ----------------------------------------------------------------------
 // Generic-proxy writes to shared memory -> visible to the async proxy (TMA, tensor core reads).
 __device__ __forceinline__ void fence_proxy_async_smem() {
