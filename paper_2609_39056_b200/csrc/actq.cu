@@ -188,6 +188,11 @@ __global__ void __launch_bounds__(1024) actq_int_row_kernel(ActqArgs a, int qmax
     const int T = blockDim.x;
     const int n_chunks = a.K >> 3;
     const float qmaxf = static_cast<float>(qmax);
+    // Let a dependent GEMM launched with programmatic dependent launch start its own set-up now; it
+    // still waits for this whole grid to finish before it reads anything written here.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (blockIdx.x == 0 && a.zero_ints != nullptr)
+        for (int i = t; i < a.n_zero; i += T) a.zero_ints[i] = 0;
 
     float dd[NCH][8];
 #pragma unroll
@@ -435,6 +440,21 @@ static int row_grid(int rows, int threads) {
     const int per_sm = 2048 / threads > 0 ? 2048 / threads : 1;
     const int cap = 148 * (per_sm > 8 ? 8 : per_sm);
     return rows < cap ? rows : cap;
+}
+
+// The GEMMs that follow these kernels use ~200 KB of shared memory.  Asking for the same carve-out here
+// keeps the SM's L1 / shared-memory split from being reconfigured at every kernel boundary.
+cudaError_t actq_init()
+{
+    cudaError_t e;
+#define RUDDER_CARVE(K)                                                                                         \
+    e = cudaFuncSetAttribute(K, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared); \
+    if (e != cudaSuccess) return e;
+    RUDDER_CARVE(actq_int_row_kernel<1>) RUDDER_CARVE(actq_int_row_kernel<2>) RUDDER_CARVE(actq_int_row_kernel<4>)
+    RUDDER_CARVE(actq_int_kernel<0>)
+    RUDDER_CARVE(actq_nvfp4_row_kernel<1>) RUDDER_CARVE(actq_nvfp4_row_kernel<2>) RUDDER_CARVE(actq_nvfp4_kernel<0>)
+#undef RUDDER_CARVE
+    return cudaSuccess;
 }
 
 cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st)

@@ -68,7 +68,7 @@ rudder_status ensure_init()
     if (cudaGetDevice(&dev) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (dev < 0 || dev >= 64) return RUDDER_ERR_CUDA;
     if (!g_gemm_ready[dev]) {
-        if (gemm_i8_init() != cudaSuccess || gemm_fp4_init() != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (gemm_i8_init() != cudaSuccess || gemm_fp4_init() != cudaSuccess || actq_init() != cudaSuccess) return RUDDER_ERR_CUDA;
         g_gemm_ready[dev] = true;
     }
     return RUDDER_OK;
@@ -110,7 +110,7 @@ size_t workspace_bytes_for(const rudder_weight* w, int M)
         return codes + sf + r;
     }
     const size_t codes = align_up(static_cast<size_t>(M) * w->K, 256);
-    return codes + r;
+    return codes + r + gemm_i8_scratch_bytes(M, w->N, w->K, false, nullptr);
 }
 
 rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M, const rudder_segments* seg,
@@ -135,6 +135,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     if (s != RUDDER_OK) return s;
 
     ActqArgs a;
+    a.zero_ints = nullptr; a.n_zero = 0;
     a.X = X; a.ldx = ldx; a.M = M; a.K = w->K; a.dinv = w->dinv;
     a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
     a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;
@@ -170,11 +171,22 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
 
     int8_t* codes = static_cast<int8_t*>(workspace);
     float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
+    const GemmI8Plan plan = gemm_i8_plan(M, w->N, w->K, acc != nullptr);
+    GemmI8Args g;
+    g.partials = nullptr; g.counters = nullptr;
+    if (plan.splitk > 1) {
+        size_t counters_off = 0;
+        gemm_i8_scratch_bytes(M, w->N, w->K, false, &counters_off);
+        uint8_t* scratch = reinterpret_cast<uint8_t*>(r) + align_up(static_cast<size_t>(M) * sizeof(float), 256);
+        g.partials = reinterpret_cast<float*>(scratch);
+        g.counters = reinterpret_cast<int*>(scratch + counters_off);
+        a.zero_ints = g.counters;
+        a.n_zero = ((M + plan.token_tile - 1) / plan.token_tile) * ((w->N + 127) / 128);
+    }
     if (launch_actq_int(a, qmax_of(w->scheme), codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
 
-    GemmI8Args g;
-    const int tt = gemm_i8_token_tile(M);
+    const int tt = plan.token_tile;
     const uint32_t box_tok = static_cast<uint32_t>(M < tt ? M : tt);
     if (!make_tmap_2d(&g.tm_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes, static_cast<uint64_t>(w->K), static_cast<uint64_t>(M),
                       static_cast<uint64_t>(w->K), 128, box_tok, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -481,6 +493,7 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
     if (s != RUDDER_OK) return s;
     if (!aligned(X, 16) || ldx % 8 != 0 || ldx < w->K || !aligned(codes, 16)) return RUDDER_ERR_ALIGN;
     ActqArgs a;
+    a.zero_ints = nullptr; a.n_zero = 0;
     a.X = X; a.ldx = ldx; a.M = M; a.K = w->K; a.dinv = w->dinv;
     a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
     a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;

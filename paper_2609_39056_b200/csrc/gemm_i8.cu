@@ -19,14 +19,23 @@
 //   warps 8-15    epilogue: per weight group, drain the INT32 partial sums from TMEM and accumulate
 //                 fp32(C) * Delta_W[j,g] in registers; finally * r_i + b_j -> bf16, transposed through
 //                 shared memory and written with one TMA store per tile.
-// Group partials alternate between two TMEM buffers, so the tensor core runs group g + 1 while group
-// g is drained.
+// Group partials rotate through the TMEM buffers, so the tensor core runs ahead of the drain (by one
+// group with 256-token tiles, by up to seven with small tiles, where the hand-shake latency per group
+// would otherwise dominate).
 //
 // Shared memory rings (stage = 128 input channels):
 //   X  [SX][TT tokens][128 B]     int8, swizzled by TMA       full: TMA bytes     empty: umma commit
 //   W  [SW][128 channels][128 B]  int8 x16, swizzled by hand  full: 4 warps       empty: umma commit
 // The output tile [TT tokens][128 channels] bf16 is staged over the X ring once the last MMA is done.
-// TMEM: 2 x TT columns x 128 lanes of INT32.  acc_full[b]: umma commit; acc_empty[b]: 8 epilogue warps.
+// Small M (action / proprio-only passes): the token tile shrinks to 32 / 64 / 128 and the K dimension
+// is split over blockIdx.y so that about one CTA per SM streams its own slice of the weights, several
+// stages of packed weights in flight per thread.  Each split writes its fp32 partial tile; the CTA that
+// arrives last at the tile's counter adds the partials in split order (deterministic) and runs the
+// normal output path.  The kernel may be launched with programmatic dependent launch: everything that
+// does not read the prologue's output (barrier set-up, TMEM allocation, weight prefetch) then overlaps
+// the prologue kernel.
+// TMEM: NBUF = 512 / TT (at most 8) buffers of TT columns x 128 lanes of INT32, one weight group each.
+// acc_full[b]: umma commit; acc_empty[b]: 8 epilogue warps.
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -75,15 +84,18 @@ constexpr int EPI_THREADS = 256;
 #define RUDDER_SLEEP_EPI 0
 #endif
 
-template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256 or 128
-    static constexpr int SX = (TT == 256) ? 4 : 6;
+template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256, 128, 64 or 32
+    static constexpr int SX = (TT == 256) ? 4 : (TT == 128) ? 6 : 8;
+    static constexpr int PD = (TT <= 64) ? 4 : (TT == 128 ? 2 : 1);   // stages of packed weights a thread keeps in flight
     static constexpr int X_BYTES = TT * KSTAGE;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + SX * X_BYTES;
     static constexpr int BYTES = OFF_W + SW * W_BYTES;
     static constexpr int DYN_SMEM = BYTES + 1024;    // slack to align the base to 1024 bytes
-    static constexpr int TMEM_COLS = 2 * TT;
+    static constexpr int NBUF = (512 / TT > 8) ? 8 : 512 / TT;   // TMEM accumulator buffers (one weight group each)
+    static constexpr int TMEM_COLS = NBUF * TT;
     static constexpr int EC = TT / 2;                // tokens per epilogue thread
+    static constexpr int CH = (EC < 32) ? EC : 32;   // tokens per TMEM load
     static_assert(SX * X_BYTES >= TT * BN * 2, "the output tile is staged over the X ring");
 };
 
@@ -95,7 +107,12 @@ struct Params {
     const float* bias;           // [N] or nullptr
     int32_t* acc;                // accumulator dump [K/G][rows][cols] or nullptr
     int row0, rows, col0, cols;
-    int m_tiles, n_tiles;        // token tiles, channel tiles (grid = m_tiles * n_tiles CTAs)
+    int m_tiles, n_tiles;        // token tiles, channel tiles (grid.x = m_tiles * n_tiles)
+    int splitk;                  // K splits (grid.y)
+    int stages_per_split;        // 128-channel stages per split
+    float* partials;             // [splitk][N][m_tiles * TT] fp32 partial sums (splitk > 1)
+    int* counters;               // [m_tiles * n_tiles] arrivals per tile, zeroed by the prologue kernel
+    int pdl;                     // launched with programmatic dependent launch
     uint32_t x_tx;               // bytes one activation TMA box delivers
     int out_pitch;               // channels per row of the staged output tile (= TMA store box width)
 #ifdef RUDDER_ROLE_PROF
@@ -106,7 +123,7 @@ struct Params {
 #ifdef RUDDER_ROLE_PROF
 #define PROF_DECL(n) long long prof_##n = 0
 #define PROF_WAIT(n, expr) [&]() { const long long t_ = clock64(); const bool r_ = (expr); prof_##n += clock64() - t_; return r_; }()
-#define PROF_PUT(i, n) do { if (blockIdx.x == 0 && p.prof) p.prof[i] = prof_##n; } while (0)
+#define PROF_PUT(i, n) do { if (blockIdx.x == 0 && blockIdx.y == 0 && p.prof) p.prof[i] = prof_##n; } while (0)
 #else
 #define PROF_DECL(n)
 #define PROF_WAIT(n, expr) (expr)
@@ -137,6 +154,17 @@ __device__ __forceinline__ float ldg_f32_volatile(const float* p) {
     asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
     return v;
 }
+__device__ __forceinline__ float ld_f32_volatile(const float* p) {
+    float v;
+    asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float4 ld_f32x4_volatile(const float* p) {
+    float4 v;
+    asm volatile("ld.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_chunk(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld_32x32b_x32(taddr, r); }
 __device__ __forceinline__ void tmem_ld_chunk(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld_32x32b_x16(taddr, r); }
 
@@ -146,10 +174,11 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 {
     using T = Tile<TT>;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * SW + 5];
+    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * SW + 2 * T::NBUF + 1];
     __shared__ __align__(16) float rs_smem[TT];      // row scales r_i of the tile's tokens (0 past M)
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_word;
+    __shared__ int last_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -157,8 +186,13 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     tile_coords(blockIdx.x, p.m_tiles, p.n_tiles, 16, tile_m, tile_n);
     const int m0 = tile_m * TT;              // first token of the tile
     const int n0 = tile_n * BN;              // first output channel of the tile
-    const int n_stages = p.K / KSTAGE;
-    const int n_groups = p.K / p.G;
+    // this CTA's share of K: stages [s0, s0 + n_stages), weight groups [g0, g0 + n_groups)
+    const int n_stages = p.stages_per_split;
+    const int s0 = blockIdx.y * n_stages;
+    const int k_split = n_stages * KSTAGE;
+    const int g_len = p.G < k_split ? p.G : k_split;     // a group longer than the split is cut: its partial
+    const int n_groups = k_split / g_len;                // integer sums are scaled and added per split
+    const int g0 = (s0 * KSTAGE) / p.G;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bar0 = smem_u32(bars);
@@ -167,14 +201,14 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     auto w_full = [&](int i) { return bar0 + 8u * (2 * T::SX + i); };
     auto w_empty = [&](int i) { return bar0 + 8u * (2 * T::SX + SW + i); };
     auto acc_full = [&](int i) { return bar0 + 8u * (2 * T::SX + 2 * SW + i); };
-    auto acc_empty = [&](int i) { return bar0 + 8u * (2 * T::SX + 2 * SW + 2 + i); };
-    const uint32_t rs_full = bar0 + 8u * (2 * T::SX + 2 * SW + 4);
+    auto acc_empty = [&](int i) { return bar0 + 8u * (2 * T::SX + 2 * SW + T::NBUF + i); };
+    const uint32_t rs_full = bar0 + 8u * (2 * T::SX + 2 * SW + 2 * T::NBUF);
 
     if (threadIdx.x == 0) {
         abort_word = 0;
         for (int i = 0; i < T::SX; ++i) { mbar_init(x_full(i), 1); mbar_init(x_empty(i), 1); }
         for (int i = 0; i < SW; ++i) { mbar_init(w_full(i), UNPACK_THREADS / 32); mbar_init(w_empty(i), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(acc_full(i), 1); mbar_init(acc_empty(i), EPI_THREADS / 32); }
+        for (int i = 0; i < T::NBUF; ++i) { mbar_init(acc_full(i), 1); mbar_init(acc_empty(i), EPI_THREADS / 32); }
         mbar_init(rs_full, 1);
         fence_mbar_init();
     }
@@ -191,12 +225,13 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     if (warp < 8) {
     // The epilogue warpgroups hold TT/2 fp32 accumulators per thread: hand them the registers the
     // producer / MMA / unpack warpgroups do not need.
-    if (TT == 256) reg_dec<RUDDER_REGS_LO>(); else reg_dec<RUDDER_REGS_LO128>();
+    if (TT == 256) reg_dec<RUDDER_REGS_LO>(); else if (TT == 128) reg_dec<RUDDER_REGS_LO128>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (activations)
         if (lane == 0) {
             tma_prefetch_desc(&tm_x);
             tma_prefetch_desc(&tm_y);
+            if (p.pdl) griddep_wait();                 // the activation codes come from the prologue kernel
             int issued = 0;
             bool ok = true;
             PROF_DECL(x_empty);
@@ -206,11 +241,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 ok = PROF_WAIT(x_empty, mbar_wait<RUDDER_SLEEP_PROD>(x_empty(slot), ph ^ 1u, abortp, W_X_EMPTY));
                 if (!ok) break;
                 mbar_expect_tx(x_full(slot), p.x_tx);
-#ifndef RUDDER_DBG_NO_TMA
-                tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, s * KSTAGE, m0, x_full(slot));
-#else
-                asm volatile("mbarrier.complete_tx.shared::cta.b64 [%0], %1;" ::"r"(x_full(slot)), "r"(p.x_tx) : "memory");
-#endif
+                tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, (s0 + s) * KSTAGE, m0, x_full(slot));
                 ++issued;
                 if (++slot == T::SX) { slot = 0; ph ^= 1u; }
             }
@@ -235,9 +266,10 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #endif
             // No divisions in this loop: every instruction on this path is latency the tensor core may
             // end up waiting for.
-            const int mma_per_group = p.G >> 5;        // MMAs (K = 32 each) per weight group
+            const int mma_per_group = g_len >> 5;      // MMAs (K = 32 each) per weight group
             int in_group = 0;                          // MMAs issued so far in the current group
-            uint32_t g = 0;                            // current group
+            uint32_t buf = 0, phb = 0;                 // accumulator buffer of the current group, its phase
+            int g_issued = 0;                          // groups started so far
             int sx = 0, sw = 0;                        // ring slots
             uint32_t phx = 0, phw = 0;                 // ring phases
             for (int s = 0; s < n_stages && ok; ++s) {
@@ -250,20 +282,18 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 const uint64_t db = umma_desc_sw128(smem_base + T::OFF_X + sx * T::X_BYTES);     // tokens: N side
 #pragma unroll
                 for (int kk = 0; kk < KSTAGE / 32; ++kk) {
-                    const uint32_t buf = g & 1u;
-                    if (in_group == 0) {
-                        ok = PROF_WAIT(acc_empty, mbar_wait<RUDDER_SLEEP_MMA>(acc_empty(buf), ((g >> 1) & 1u) ^ 1u, abortp, W_ACC_EMPTY));
+                    if (in_group == 0 && g_issued >= T::NBUF) {     // a buffer's first use needs no wait
+                        ok = PROF_WAIT(acc_empty, mbar_wait<RUDDER_SLEEP_MMA>(acc_empty(buf), phb ^ 1u, abortp, W_ACC_EMPTY));
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                         tcgen05_fence_after_sync();
                     }
-#ifndef RUDDER_DBG_NO_MMA
                     if (leader) umma_i8(tmem_base + buf * TT, da + 2u * kk, db + 2u * kk, idesc, in_group == 0 ? 0u : 1u);
-#endif
                     if (++in_group == mma_per_group) {
                         if (leader) umma_commit(acc_full(buf));
                         in_group = 0;
-                        ++g;
+                        ++g_issued;
+                        if (++buf == T::NBUF) { buf = 0; phb ^= 1u; }
                     }
                 }
                 if (!ok) break;
@@ -282,7 +312,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ row scales of the tile -> shared
-        for (int i = lane; i < TT; i += 32) rs_smem[i] = (m0 + i < p.M) ? __ldg(p.row_scale + m0 + i) : 0.0f;
+        if (p.pdl) griddep_wait();                     // so do the row scales
+        for (int i = lane; i < TT; i += 32) rs_smem[i] = (m0 + i < p.M) ? ld_f32_volatile(p.row_scale + m0 + i) : 0.0f;
         __syncwarp();
         if (lane == 0) mbar_arrive(rs_full);
     } else if (warp >= 4) {
@@ -304,44 +335,54 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             valid[i] = (n0 + row) < p.N;
             src[i] = p.codes + static_cast<size_t>(valid[i] ? n0 + row : 0) * row_bytes + ch * 16;
         }
-        uint4 nxt[4];
+        // PD stages of packed weights are in flight per thread (registers), so that the L2 / DRAM latency
+        // of the weight stream is covered even when a stage is consumed quickly.
+        constexpr int PD = T::PD;
+        uint4 pre[PD][4];
+        auto load_stage = [&](int s, uint4 (&dst)[4]) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) nxt[i] = valid[i] ? ldg_nc_16(src[i]) : make_uint4(0, 0, 0, 0);
-        for (int s = 0; s < n_stages; ++s) {
-            uint4 cur[4];
+            for (int i = 0; i < 4; ++i)
+                dst[i] = valid[i] ? ldg_nc_16(src[i] + static_cast<size_t>(s0 + s) * (KSTAGE / 2)) : make_uint4(0, 0, 0, 0);
+        };
 #pragma unroll
-            for (int i = 0; i < 4; ++i) cur[i] = nxt[i];
-            if (s + 1 < n_stages) {
+        for (int j = 0; j < PD; ++j)
+            if (j < n_stages) load_stage(j, pre[j]);
+        bool ok = true;
+        int sw = 0;
+        uint32_t phw = 0;
+        for (int sb = 0; sb < n_stages && ok; sb += PD) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    nxt[i] = valid[i] ? ldg_nc_16(src[i] + static_cast<size_t>(s + 1) * (KSTAGE / 2)) : make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < PD; ++j) {
+                const int s = sb + j;
+                if (s < n_stages && ok) {
+                    uint4 cur[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) cur[i] = pre[j][i];
+                    if (s + PD < n_stages) load_stage(s + PD, pre[j]);
+                    ok = PROF_WAIT(w_empty, mbar_wait<RUDDER_SLEEP_UNPACK>(w_empty(sw), phw ^ 1u, abortp, W_W_EMPTY));
+                    if (ok) {
+                        const uint32_t dst = smem_base + T::OFF_W + sw * W_BYTES;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int idx = i * UNPACK_THREADS + tid;
+                            const int row = idx >> 2, ch = idx & 3;
+                            const uint4 pk = cur[i];
+                            uint4 lo, hi;
+                            lo.x = (pk.x << 4) & 0xF0F0F0F0u; hi.x = pk.x & 0xF0F0F0F0u;
+                            lo.y = (pk.y << 4) & 0xF0F0F0F0u; hi.y = pk.y & 0xF0F0F0F0u;
+                            lo.z = (pk.z << 4) & 0xF0F0F0F0u; hi.z = pk.z & 0xF0F0F0F0u;
+                            lo.w = (pk.w << 4) & 0xF0F0F0F0u; hi.w = pk.w & 0xF0F0F0F0u;
+                            const uint32_t drow = dst + (row >> 3) * 1024 + (row & 7) * 128;
+                            sts128(drow + (((2 * ch) ^ (row & 7)) << 4), lo);
+                            sts128(drow + (((2 * ch + 1) ^ (row & 7)) << 4), hi);
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(w_full(sw));      // one arrival per warp: arrivals on one barrier serialise
+                        if (++sw == SW) { sw = 0; phw ^= 1u; }
+                    }
+                }
             }
-            const int sw = s % SW;
-            if (!PROF_WAIT(w_empty, mbar_wait<RUDDER_SLEEP_UNPACK>(w_empty(sw), ((s / SW) & 1) ^ 1, abortp, W_W_EMPTY))) break;
-            const uint32_t dst = smem_base + T::OFF_W + sw * W_BYTES;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int idx = i * UNPACK_THREADS + tid;
-                const int row = idx >> 2, ch = idx & 3;
-                const uint4 pk = cur[i];
-                uint4 lo, hi;
-                lo.x = (pk.x << 4) & 0xF0F0F0F0u; hi.x = pk.x & 0xF0F0F0F0u;
-                lo.y = (pk.y << 4) & 0xF0F0F0F0u; hi.y = pk.y & 0xF0F0F0F0u;
-                lo.z = (pk.z << 4) & 0xF0F0F0F0u; hi.z = pk.z & 0xF0F0F0F0u;
-                lo.w = (pk.w << 4) & 0xF0F0F0F0u; hi.w = pk.w & 0xF0F0F0F0u;
-                const uint32_t drow = dst + (row >> 3) * 1024 + (row & 7) * 128;
-#ifndef RUDDER_DBG_NO_STS
-                sts128(drow + (((2 * ch) ^ (row & 7)) << 4), lo);
-                sts128(drow + (((2 * ch + 1) ^ (row & 7)) << 4), hi);
-#else
-                if (lo.x == 0x12345678u && hi.y == 0x9abcdef0u) sts128(drow, lo);
-#endif
-            }
-#ifndef RUDDER_DBG_NO_FENCE
-            fence_proxy_async_smem();
-#endif
-            __syncwarp();
-            if (lane == 0) mbar_arrive(w_full(sw));      // one arrival per warp: arrivals on one barrier serialise
         }
 #ifdef RUDDER_ROLE_PROF
         prof_unpack_total = clock64() - un_t0;
@@ -350,9 +391,9 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     }
     } else {
         // ------------------------------------------------------------------ epilogue
-        if (TT == 256) reg_inc<RUDDER_REGS_HI>(); else reg_inc<RUDDER_REGS_HI128>();
+        if (TT == 256) reg_inc<RUDDER_REGS_HI>(); else if (TT == 128) reg_inc<RUDDER_REGS_HI128>();
         constexpr int EC = T::EC;
-        constexpr int CH = (TT == 256) ? RUDDER_CH : 32;   // tokens per TMEM load
+        constexpr int CH = T::CH;                // tokens per TMEM load
         constexpr int NCH = EC / CH;
         const int q = warp & 3;                  // TMEM lane quadrant this warp may read
         const int h = (warp - 8) >> 2;           // token half
@@ -369,28 +410,68 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #endif
         // Scales are fetched two groups ahead with volatile loads: a plain load would be sunk next to
         // its use and expose the L2 latency once per group.
-        const float* sc_ptr = p.scales_t + (n_ok ? n : 0);
+        const float* sc_ptr = p.scales_t + static_cast<size_t>(g0) * p.N + (n_ok ? n : 0);
         float sc_next = ldg_f32_volatile(sc_ptr);
         float sc_next2 = (n_groups > 1) ? ldg_f32_volatile(sc_ptr + p.N) : 0.0f;
-        for (int g = 0; g < n_groups; ++g) {
-            const int buf = g & 1;
-#ifdef RUDDER_DBG_CONST_SC
-            const float sc = 1.5f + threadIdx.x;
-#else
+        int buf = 0;
+        uint32_t phb = 0;
+        int g = 0;
+        if (NCH == 1 && !DUMP) {
+            // Small tiles: a group is one TMEM load per thread, so the fixed cost of a hand-shake (barrier
+            // poll, vote, fences) dominates.  Take up to four groups per round: poll their barriers, issue
+            // all the loads, wait once, then scale and accumulate.
+            constexpr int GU = (T::NBUF >= 4) ? 4 : T::NBUF;
+            for (; g + GU <= n_groups && ok; g += GU) {
+                float scu[GU];
+#pragma unroll
+                for (int u = 0; u < GU; ++u) scu[u] = n_ok ? ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + u) * p.N) : 0.0f;
+                if (lane == 0) {
+#pragma unroll
+                    for (int u = 0; u < GU; ++u)
+                        ok = ok && mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf + u), phb, abortp, W_ACC_FULL);
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                tcgen05_fence_after_sync();
+                uint32_t c[GU][CH];
+#pragma unroll
+                for (int u = 0; u < GU; ++u)
+                    tmem_ld_chunk(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (buf + u) * TT + h * EC, c[u]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int u = 0; u < GU; ++u) {
+                    float f[CH];
+#pragma unroll
+                    for (int j = 0; j < CH; ++j) asm volatile("cvt.rn.f32.s32 %0, %1;" : "=f"(f[j]) : "r"(c[u][j]));
+#pragma unroll
+                    for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[j]) : "f"(f[j]), "f"(scu[u]));
+                }
+                tcgen05_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+#pragma unroll
+                    for (int u = 0; u < GU; ++u) mbar_arrive(acc_empty(buf + u));
+                }
+                buf += GU;                               // NBUF is a multiple of GU: no wrap inside a round
+                if (buf == T::NBUF) { buf = 0; phb ^= 1u; }
+            }
+            if (g < n_groups) {                          // the scale prefetch of the one-group loop starts here
+                sc_next = ldg_f32_volatile(sc_ptr + static_cast<size_t>(g) * p.N);
+                sc_next2 = (g + 1 < n_groups) ? ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + 1) * p.N) : 0.0f;
+            }
+        }
+        for (; g < n_groups && ok; ++g) {
             const float sc = n_ok ? sc_next : 0.0f;
             sc_next = sc_next2;
             if (g + 2 < n_groups) sc_next2 = ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + 2) * p.N);
-#endif
-#ifndef RUDDER_DBG_EPI_FREE
             // lane 0 polls, the others wait at the shuffle: no 32-way spin, and the verdict is warp-uniform
             // (the TMEM loads below are warp-collective)
-            if (lane == 0) ok = PROF_WAIT(acc_full, mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), (g >> 1) & 1, abortp, W_ACC_FULL));
+            if (lane == 0) ok = PROF_WAIT(acc_full, mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), phb, abortp, W_ACC_FULL));
 #ifdef RUDDER_ROLE_PROF
             const long long v_t0 = clock64();
 #endif
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-#endif
 #ifdef RUDDER_ROLE_PROF
             const long long f_t0 = clock64();
             prof_epi_vote += f_t0 - v_t0;
@@ -443,7 +524,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                             const int tok = m0 + h * EC + ch * CH + j;
                             const int rr = tok - p.row0;
                             if (tok < p.M && rr >= 0 && rr < p.rows)
-                                p.acc[(static_cast<size_t>(g) * p.rows + rr) * p.cols + cc] = static_cast<int>(cur[j]) >> 4;
+                                p.acc[(static_cast<size_t>(g0 + g) * p.rows + rr) * p.cols + cc] = static_cast<int>(cur[j]) >> 4;
                         }
                     }
                 }
@@ -451,6 +532,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             tcgen05_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(buf));  // one arrival per warp: arrivals on one barrier serialise
+            if (++buf == T::NBUF) { buf = 0; phb ^= 1u; }
 #ifdef RUDDER_ROLE_PROF
             prof_epi_drain += clock64() - dr_t0;
 #endif
@@ -459,8 +541,41 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         prof_epi_total = clock64() - ep_t0;
         const long long tail_t0 = clock64();
 #endif
+        // Split K: publish this split's partial sums; the CTA that arrives last at the tile's counter adds
+        // the splits in order and goes on to write the tile, the others are done.
+        bool writer = true;
+        if (TT <= 128 && p.splitk > 1) {           // only small-M launches split K
+            const int m_pad = p.m_tiles * TT;
+            float* mine = p.partials + (static_cast<size_t>(blockIdx.y) * p.N + (n_ok ? n : 0)) * m_pad + m0 + h * EC;
+            if (ok && n_ok) {
+#pragma unroll
+                for (int j = 0; j < EC; j += 4)
+                    *reinterpret_cast<float4*>(mine + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+            }
+            __threadfence();
+            asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+            if (threadIdx.x == 256) last_flag = (atomicAdd(p.counters + blockIdx.x, 1) == p.splitk - 1) ? 1 : 0;
+            asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+            writer = last_flag != 0;
+            if (writer && ok) {
+                __threadfence();
+#pragma unroll
+                for (int j = 0; j < EC; ++j) acc[j] = 0.0f;
+                if (n_ok) {
+                    for (int z = 0; z < p.splitk; ++z) {
+                        const float* src = p.partials + (static_cast<size_t>(z) * p.N + n) * m_pad + m0 + h * EC;
+#pragma unroll
+                        for (int j = 0; j < EC; j += 4) {
+                            const float4 v = ld_f32x4_volatile(src + j);
+                            acc[j] += v.x; acc[j + 1] += v.y; acc[j + 2] += v.z; acc[j + 3] += v.w;
+                        }
+                    }
+                }
+            }
+        }
         // The last acc_full arrives after every MMA of the tile has completed, so the X ring is free:
         // stage the transposed bf16 tile there ([token][channel], `out_pitch` channels per row).
+        ok = ok && writer;
         if (ok) ok = mbar_wait<64>(rs_full, 0, abortp, W_RS_FULL);
         if (ok) {
             const float b = (p.bias != nullptr && n_ok) ? __ldg(p.bias + n) : 0.0f;
@@ -506,7 +621,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 }  // namespace
 
 template <int TT, bool DUMP>
-static cudaError_t launch_one(const GemmI8Args& a, cudaStream_t st)
+static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaStream_t st)
 {
     using T = Tile<TT>;
     Params p;
@@ -522,33 +637,92 @@ static cudaError_t launch_one(const GemmI8Args& a, cudaStream_t st)
 #endif
     p.m_tiles = (a.M + TT - 1) / TT;
     p.n_tiles = (a.N + BN - 1) / BN;
-    gemm_i8_w4_kernel<TT, DUMP><<<p.m_tiles * p.n_tiles, NUM_THREADS, T::DYN_SMEM, st>>>(a.tm_x, a.tm_y, p);
-    return cudaGetLastError();
+    p.splitk = plan.splitk;
+    p.stages_per_split = a.K / KSTAGE / plan.splitk;
+    p.partials = a.partials;
+    p.counters = a.counters;
+    p.pdl = plan.pdl ? 1 : 0;
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.m_tiles * p.n_tiles, plan.splitk, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = T::DYN_SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = plan.pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_kernel<TT, DUMP>, a.tm_x, a.tm_y, p);
 }
 
-int gemm_i8_token_tile(int M) { return M > 128 ? 256 : 128; }
+// Tile and split choice.  Large M: 256-token tiles, no split.  M <= 256: the smallest tile that holds
+// the rows, and K split so that about one CTA per SM streams weights, as long as every split keeps at
+// least two stages and the fp32 partials stay small (they must also fit the fixed scratch of
+// rudder_linear_static).
+GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump)
+{
+    GemmI8Plan plan;
+    plan.token_tile = M > 128 ? 256 : (M > 64 ? 128 : (M > 32 ? 64 : 32));
+    plan.splitk = 1;
+    plan.pdl = false;
+#ifdef RUDDER_ROLE_PROF
+    dump = false;               // development build: the dump pointer carries cycle counters, not accumulators
+#endif
+    if (dump || M > 256) return plan;
+    const int n_tiles = (N + BN - 1) / BN;
+    if (M > 128 && n_tiles < 74) plan.token_tile = 128;       // two token tiles double the CTAs
+    const int m_tiles = (M + plan.token_tile - 1) / plan.token_tile;
+    const int base = m_tiles * n_tiles;
+    const size_t m_pad = static_cast<size_t>(m_tiles) * plan.token_tile;
+    int sk = 1;
+    while (sk < 16 && base * (sk * 2) <= 160 && (K / KSTAGE) % (sk * 2) == 0 && K / (sk * 2) >= 2 * KSTAGE &&
+           static_cast<size_t>(sk * 2) * N * m_pad * sizeof(float) <= (size_t(2) << 20))
+        sk *= 2;
+    plan.splitk = sk;
+    plan.pdl = true;
+    return plan;
+}
+
+size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_offset)
+{
+    const GemmI8Plan plan = gemm_i8_plan(M, N, K, dump);
+    const int n_tiles = (N + BN - 1) / BN;
+    const int m_tiles = (M + plan.token_tile - 1) / plan.token_tile;
+    size_t partial = 0;
+    if (plan.splitk > 1) partial = static_cast<size_t>(plan.splitk) * N * m_tiles * plan.token_tile * sizeof(float);
+    partial = (partial + 255) / 256 * 256;
+    if (counters_offset) *counters_offset = partial;
+    const size_t counters = plan.splitk > 1 ? (static_cast<size_t>(m_tiles) * n_tiles * sizeof(int) + 255) / 256 * 256 : 0;
+    return partial + counters;
+}
 
 cudaError_t gemm_i8_init()
 {
     cudaError_t e;
-    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<128>::DYN_SMEM);
+#define RUDDER_I8_ATTR(TT, D)                                                                                          \
+    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT>::DYN_SMEM); \
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<128>::DYN_SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<256>::DYN_SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<256>::DYN_SMEM);
-    return e;
+    RUDDER_I8_ATTR(32, false) RUDDER_I8_ATTR(64, false) RUDDER_I8_ATTR(128, false) RUDDER_I8_ATTR(256, false)
+    RUDDER_I8_ATTR(32, true) RUDDER_I8_ATTR(64, true) RUDDER_I8_ATTR(128, true) RUDDER_I8_ATTR(256, true)
+#undef RUDDER_I8_ATTR
+    return cudaSuccess;
 }
 
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st)
 {
-    const bool wide = gemm_i8_token_tile(a.M) == 256;
+    const GemmI8Plan plan = gemm_i8_plan(a.M, a.N, a.K, a.acc != nullptr);
 #ifdef RUDDER_ROLE_PROF
-    return wide ? launch_one<256, false>(a, st) : launch_one<128, false>(a, st);   // the dump pointer carries counters
+    const bool dump = false;                        // the dump pointer carries counters in this build
+#else
+    const bool dump = a.acc != nullptr;
 #endif
-    if (a.acc != nullptr) return wide ? launch_one<256, true>(a, st) : launch_one<128, true>(a, st);
-    return wide ? launch_one<256, false>(a, st) : launch_one<128, false>(a, st);
+    switch (plan.token_tile) {
+        case 32:  return dump ? launch_one<32, true>(a, plan, st) : launch_one<32, false>(a, plan, st);
+        case 64:  return dump ? launch_one<64, true>(a, plan, st) : launch_one<64, false>(a, plan, st);
+        case 128: return dump ? launch_one<128, true>(a, plan, st) : launch_one<128, false>(a, plan, st);
+        default:  return dump ? launch_one<256, true>(a, plan, st) : launch_one<256, false>(a, plan, st);
+    }
 }
 
 }  // namespace rudder

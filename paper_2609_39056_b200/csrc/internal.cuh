@@ -48,6 +48,8 @@ struct rudder_weight {
 namespace rudder {
 
 struct ActqArgs {
+    int* zero_ints;            // words the kernel clears for the GEMM that follows (tile counters), or nullptr
+    int n_zero;
     const uint16_t* X;
     int64_t ldx;
     int M, K;
@@ -63,6 +65,7 @@ cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G
                              cudaStream_t st);
 cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, cudaStream_t st);
 
+cudaError_t actq_init();
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);
 cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st);
 cudaError_t launch_pack_nvfp4(const float* W, const float* d, int N, int K, uint8_t* codes, uint8_t* sb_canonical,
@@ -97,8 +100,16 @@ struct GemmI8Args {
     // accumulator dump (parity hook); acc == nullptr in production
     int32_t* acc;
     int row0, rows, col0, cols;
+    float* partials;            // split-K scratch (see gemm_i8_scratch_bytes) or nullptr
+    int* counters;              // per-tile arrival counters, zeroed by the prologue kernel, or nullptr
 };
-int gemm_i8_token_tile(int M);  // tokens per CTA tile the GEMM will use for M rows (sizes the TMA boxes)
+struct GemmI8Plan {
+    int token_tile;             // tokens per CTA tile: sizes the TMA boxes
+    int splitk;                 // K splits
+    bool pdl;                   // launched with programmatic dependent launch after the prologue kernel
+};
+GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump);
+size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_offset);
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st);
 cudaError_t gemm_i8_init();     // one-time function attributes (dynamic shared memory opt-in)
 
