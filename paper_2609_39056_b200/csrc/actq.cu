@@ -10,6 +10,10 @@
 #include "internal.cuh"
 #include "fp4.cuh"
 
+#ifndef RUDDER_ROW_NCH
+#define RUDDER_ROW_NCH 2            // blocks of 16 channels per thread of the row kernels
+#endif
+
 namespace rudder {
 
 __device__ __forceinline__ uint4 ld_nc_16(const uint4* p) {
@@ -129,123 +133,6 @@ __global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int
         r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, static_cast<float>(qmax)), g) : 0.0f;
 }
 
-// ---- one row per CTA step ------------------------------------------------------------------------
-// The warp-per-row kernels above keep a whole row in one warp's registers, which caps the occupancy and
-// leaves the memory system idle while a warp computes.  Here a row is spread over the T threads of a
-// CTA (T = row pieces, up to 1024; NCH pieces per thread for longer rows).  The CTA is persistent: it
-// walks rows blockIdx.x, blockIdx.x + gridDim.x, ..., so a thread always meets the same input channels
-// and keeps their dinv in registers, and it issues the loads of its next row before working on the
-// current one.  Range pass: max_k |x dinv| and one multiplication by gamma -- identical bits to
-// max_k |(x dinv) gamma| because rounding is monotonic and gamma > 0.
-__device__ __forceinline__ float block_max(float m, float* red /* [32] shared */) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    const int n_warps = (blockDim.x + 31) >> 5;
-    if (n_warps == 1) return m;
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
-    __syncthreads();
-    float r = (static_cast<int>(threadIdx.x & 31) < n_warps) ? red[threadIdx.x & 31] : 0.0f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xffffffffu, r, o));
-    return r;
-}
-
-// x (8 bf16) * dinv -> 8 fp32 (the first of the two roundings of v = (x dinv) gamma)
-__device__ __forceinline__ void mul_dinv8(const uint4& x, const float (&dd)[8], float (&u)[8]) {
-    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        u[2 * i] = __fmul_rn(__uint_as_float(w[i] << 16), dd[2 * i]);
-        u[2 * i + 1] = __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), dd[2 * i + 1]);
-    }
-}
-
-// Eight scaled values -> eight int8 codes.  CLAMP: static range (values may exceed the range).
-template <bool CLAMP>
-__device__ __forceinline__ uint2 round8_fast(const float (&v)[8], float inv, float qmaxf) {
-    int q[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        float t = __fmul_rn(v[i], inv);
-        if (CLAMP) t = fminf(fmaxf(t, -qmaxf), qmaxf);
-        q[i] = __float2int_rn(t);
-    }
-    uint32_t lo, hi, t0, t1;
-    // cvt.pack: two s32 -> two saturated s8 in the low half, third operand supplies the upper half
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(t0) : "r"(q[3]), "r"(q[2]));
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(lo) : "r"(q[1]), "r"(q[0]), "r"(t0));
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(t1) : "r"(q[7]), "r"(q[6]));
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q[5]), "r"(q[4]), "r"(t1));
-    return make_uint2(lo, hi);
-}
-
-template <int NCH>
-__global__ void __launch_bounds__(1024) actq_int_row_kernel(ActqArgs a, int qmax, int8_t* __restrict__ codes, int64_t ldc,
-                                                             float* __restrict__ r)
-{
-    __shared__ float red[2][32];
-    const int t = threadIdx.x;
-    const int T = blockDim.x;
-    const int n_chunks = a.K >> 3;
-    const float qmaxf = static_cast<float>(qmax);
-    // Let a dependent GEMM launched with programmatic dependent launch start its own set-up now; it
-    // still waits for this whole grid to finish before it reads anything written here.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (blockIdx.x == 0 && a.zero_ints != nullptr)
-        for (int i = t; i < a.n_zero; i += T) a.zero_ints[i] = 0;
-
-    float dd[NCH][8];
-#pragma unroll
-    for (int i = 0; i < NCH; ++i) {
-        const int c = i * T + t;
-        const float4 d0 = (c < n_chunks) ? __ldg(reinterpret_cast<const float4*>(a.dinv) + 2 * c) : make_float4(0, 0, 0, 0);
-        const float4 d1 = (c < n_chunks) ? __ldg(reinterpret_cast<const float4*>(a.dinv) + 2 * c + 1) : make_float4(0, 0, 0, 0);
-        dd[i][0] = d0.x; dd[i][1] = d0.y; dd[i][2] = d0.z; dd[i][3] = d0.w;
-        dd[i][4] = d1.x; dd[i][5] = d1.y; dd[i][6] = d1.z; dd[i][7] = d1.w;
-    }
-    auto load_row = [&](int row, uint4 (&x)[NCH]) {
-        const bool live = row < a.M;
-        const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(live ? row : 0) * a.ldx);
-#pragma unroll
-        for (int i = 0; i < NCH; ++i) {
-            const int c = i * T + t;
-            x[i] = (live && c < n_chunks) ? ld_nc_16(xrow + c) : make_uint4(0, 0, 0, 0);
-        }
-    };
-
-    uint4 nxt[NCH];
-    load_row(blockIdx.x, nxt);
-    int par = 0;
-    for (int row = blockIdx.x; row < a.M; row += gridDim.x, par ^= 1) {
-        float u[NCH][8];
-        float m = 0.0f;
-#pragma unroll
-        for (int i = 0; i < NCH; ++i) {
-            mul_dinv8(nxt[i], dd[i], u[i]);       // pieces past the row end are zero
-#pragma unroll
-            for (int j = 0; j < 8; ++j) m = fmaxf(m, fabsf(u[i][j]));
-        }
-        load_row(row + gridDim.x, nxt);            // prefetch the next row
-        const float g = a.gamma_step[stream_of_row(a.seg, row)];
-        float range;
-        if (a.clip_step == nullptr) range = __fmul_rn(block_max(m, red[par]), g);
-        else                        range = *a.clip_step;
-        const float inv = (range != 0.0f) ? __fdiv_rn(qmaxf, range) : 0.0f;
-        uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldc);
-#pragma unroll
-        for (int i = 0; i < NCH; ++i) {
-            const int c = i * T + t;
-            if (c < n_chunks) {
-                float v[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = __fmul_rn(u[i][j], g);
-                crow[c] = (a.clip_step == nullptr) ? round8_fast<false>(v, inv, qmaxf) : round8_fast<true>(v, inv, qmaxf);
-            }
-        }
-        if (t == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, qmaxf), g) : 0.0f;
-    }
-}
-
 // ---- NVFP4 activations -------------------------------------------------------------------------
 // One warp per row; a lane owns one block of 16 channels per step (two 16-byte loads), so a warp step
 // covers 512 channels.  Writes packed E2M1 codes [M, K/2], one UE4M3 scale per block (in the tensor
@@ -343,146 +230,328 @@ __global__ void __launch_bounds__(256) actq_nvfp4_kernel(ActqArgs a, int M_pad, 
         r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, kNvfp4Range), g) : 0.0f;
 }
 
-template <int NCH>
-__global__ void __launch_bounds__(1024) actq_nvfp4_row_kernel(ActqArgs a, int M_pad, uint8_t* __restrict__ codes,
-                                                               uint8_t* __restrict__ sf, int sf_tiled, float* __restrict__ r)
+// ---- one row per CTA step ------------------------------------------------------------------------
+// The warp-per-row kernels keep a whole row in one warp's registers, which caps the occupancy and
+// leaves the memory system idle while a warp computes.  Here a row is spread over the T threads of a
+// persistent CTA, NCH blocks of 16 channels per thread, and the CTA walks rows blockIdx.x,
+// blockIdx.x + gridDim.x, ...: a thread always meets the same channels and keeps their dinv in
+// registers.  Rows are staged in shared memory by bulk copies that run kRowSlots rows ahead of the
+// arithmetic (one thread issues them), so the bytes in flight do not depend on registers or occupancy.
+// Range pass: max_k |x dinv| and one multiplication by gamma -- identical bits to max_k |(x dinv) gamma|
+// because rounding is monotonic and gamma > 0.  The kernel is bound by instruction issue before it is
+// bound by HBM, so the arithmetic is kept to the fewest instructions that still round exactly like the
+// scalar definition: packed two-lane fp32 multiplies (each lane rounded on its own), one warp-wide
+// integer max instruction for the range (non-negative floats order like their bit patterns), a
+// shared-memory atomic max across warps, and a table for the reciprocal of the block scale.
+constexpr int kRowSlots = 4;
+constexpr int W_ROW_FULL = 40;                     // wait identifier reported on a timeout
+
+struct RowOut {
+    void* codes;               // int8 [M, ldc] or packed E2M1 [M, K/2]
+    int64_t ldc;               // bytes per code row
+    uint8_t* sf;               // NVFP4 block scales
+    int sf_tiled;              // tensor-core order (with zeroed padding rows up to M_pad) or row-major
+    float* r;
+    int M_pad;
+    int qmax;
+};
+
+typedef unsigned long long f32x2;                  // two fp32 lanes in one 64-bit register pair
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 p;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "f"(lo), "f"(hi));
+    return p;
+}
+__device__ __forceinline__ void unpack2(f32x2 p, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+// a *= b per lane, each product rounded to nearest on its own
+__device__ __forceinline__ void mul2(f32x2& a, f32x2 b) {
+    asm("mul.rn.f32x2 %0, %0, %1;" : "+l"(a) : "l"(b));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void bulk_row_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Maximum over the CTA of a non-negative float.  `red` holds three slots that rotate from row to row:
+// slot (i + 1) % 3 is cleared while row i is reduced; it was last read before the barrier of row i - 1,
+// which thread 0 has already passed, and is next written after the barrier of row i.
+__device__ __forceinline__ float cta_max_nonneg(float m, uint32_t* red, int& slot) {
+    const uint32_t wm = __reduce_max_sync(0xffffffffu, __float_as_uint(m));
+    const int nxt = (slot == 2) ? 0 : slot + 1;
+    if ((threadIdx.x & 31) == 0) atomicMax(red + slot, wm);
+    if (threadIdx.x == 0) red[nxt] = 0u;
+    __syncthreads();
+    const float r = __uint_as_float(*reinterpret_cast<volatile uint32_t*>(red + slot));
+    slot = nxt;
+    return r;
+}
+
+// 8 bf16 (one 16-byte word) times 8 channel scales -> 4 lane pairs; returns max |.| of the products
+__device__ __forceinline__ float mul_dinv8(const uint4& x, const f32x2* dd, f32x2* u) {
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+    float lo[4], hi[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        u[i] = pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
+        mul2(u[i], dd[i]);
+        unpack2(u[i], lo[i], hi[i]);
+    }
+    float m = fmaxf(fabsf(lo[0]), fabsf(hi[0]));
+#pragma unroll
+    for (int i = 1; i < 4; ++i) m = fmaxf(fmaxf(m, fabsf(lo[i])), fabsf(hi[i]));
+    return m;
+}
+
+// Correctly rounded a / 6 for a >= 0 (quotient, remainder by fma, one correction; checked against the
+// IEEE division for every float whose quotient is a normal number -- smaller ones encode as zero).
+__device__ __forceinline__ float div6(float a) {
+    const float c = 1.0f / 6.0f;
+    const float q0 = __fmul_rn(a, c);
+    const float rem = __fmaf_rn(-6.0f, q0, a);
+    return __fmaf_rn(rem, c, q0);
+}
+
+// Four lane pairs -> eight E2M1 codes in one word, element i in nibble i.
+__device__ __forceinline__ uint32_t e2m1x8(const f32x2* v) {
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) unpack2(v[i], f[2 * i], f[2 * i + 1]);
+    return f32x8_to_e2m1(f);
+}
+// Four lane pairs -> eight int8 codes.  CLAMP: static range (values may exceed the range).
+template <bool CLAMP>
+__device__ __forceinline__ uint2 s8x8(const f32x2* v, float qmaxf) {
+    int q[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float lo, hi;
+        unpack2(v[i], lo, hi);
+        if (CLAMP) { lo = fminf(fmaxf(lo, -qmaxf), qmaxf); hi = fminf(fmaxf(hi, -qmaxf), qmaxf); }
+        q[2 * i] = __float2int_rn(lo);
+        q[2 * i + 1] = __float2int_rn(hi);
+    }
+    uint32_t lo, hi, t0, t1;
+    // cvt.pack: two s32 -> two saturated s8 in the low half, third operand supplies the upper half
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(t0) : "r"(q[3]), "r"(q[2]));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(lo) : "r"(q[1]), "r"(q[0]), "r"(t0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(t1) : "r"(q[7]), "r"(q[6]));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q[5]), "r"(q[4]), "r"(t1));
+    return make_uint2(lo, hi);
+}
+
+template <bool FP4, int NCH>
+__global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq_row_kernel(ActqArgs a, RowOut o)
 {
-    __shared__ float red[2][32];
+    extern __shared__ __align__(128) uint8_t ring[];          // kRowSlots rows of K bf16
+    __shared__ __align__(8) uint64_t full_bar[kRowSlots];
+    __shared__ float g_slot[kRowSlots];                        // gain of the row staged in each slot
+    __shared__ uint32_t red[3];
+    __shared__ float rb_tab[128];                              // 1 / (decoded UE4M3 scale), 0 for a zero scale
+    __shared__ int abort_word;
+
     const int t = threadIdx.x;
     const int T = blockDim.x;
-    const int lane = t & 31;
+    const int M = a.M;
     const int n_blocks = a.K >> 4;
-    const int k64 = a.K >> 6;
+    const uint32_t row_bytes = static_cast<uint32_t>(a.K) * 2u;
+    const int first = blockIdx.x;
+    const int stride = gridDim.x;
+    const uint32_t ring_addr = smem_u32(ring);
+    const uint32_t bar0 = smem_u32(full_bar);
+    // Let a dependent GEMM launched with programmatic dependent launch start its own set-up now; it
+    // still waits for this whole grid to finish before it reads anything written here.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (blockIdx.x == 0 && a.zero_ints != nullptr)
+        for (int i = t; i < a.n_zero; i += T) a.zero_ints[i] = 0;
+    if (t == 0) {
+        abort_word = 0;
+        for (int i = 0; i < kRowSlots; ++i) mbar_init(bar0 + 8u * i, 1);
+        fence_mbar_init();
+    }
+    if (t < 3) red[t] = 0u;
+    if (FP4) {
+        for (int i = t; i < 128; i += T) {
+            const float sbd = ue4m3_to_f32(i);
+            rb_tab[i] = (sbd != 0.0f && i < 127) ? __fdiv_rn(1.0f, sbd) : 0.0f;
+        }
+    }
+    __syncthreads();
 
-    float dd[NCH][16];
+    // this CTA's rows: first + j * stride; j < n_live are rows of X, the rest (NVFP4, tiled scales) are
+    // the padding rows of the last 128-row scale atom, which only get zero scales
+    const int M_rows = FP4 ? o.M_pad : M;
+    const int n_rows = first < M_rows ? (M_rows - 1 - first) / stride + 1 : 0;
+    const int n_live = first < M ? (M - 1 - first) / stride + 1 : 0;
+    auto issue = [&](int j) {                                  // thread 0: stage row j of this CTA
+        const int slot = j & (kRowSlots - 1);
+        const int row = first + j * stride;
+        g_slot[slot] = __ldg(a.gamma_step + stream_of_row(a.seg, row));
+        mbar_expect_tx(bar0 + 8u * slot, row_bytes);
+        bulk_row_load(ring_addr + slot * row_bytes, a.X + static_cast<size_t>(row) * a.ldx, row_bytes, bar0 + 8u * slot);
+    };
+    if (t == 0)
+        for (int j = 0; j < kRowSlots && j < n_live; ++j) issue(j);
+
+    f32x2 dd[NCH][8];
+    uint32_t lds_off[NCH];                         // byte offset of the thread's blocks in a staged row
+    size_t sf_col[NCH];                            // column part of the scale's address
 #pragma unroll
     for (int i = 0; i < NCH; ++i) {
         const int kb = i * T + t;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const float4 d4 = (kb < n_blocks) ? __ldg(reinterpret_cast<const float4*>(a.dinv) + 4 * kb + j) : make_float4(0, 0, 0, 0);
-            dd[i][4 * j] = d4.x; dd[i][4 * j + 1] = d4.y; dd[i][4 * j + 2] = d4.z; dd[i][4 * j + 3] = d4.w;
+            dd[i][2 * j] = pack2(d4.x, d4.y);
+            dd[i][2 * j + 1] = pack2(d4.z, d4.w);
         }
+        lds_off[i] = static_cast<uint32_t>(kb < n_blocks ? kb : n_blocks - 1) * 32u;   // spare threads re-read the last block (their dinv is 0)
+        sf_col[i] = o.sf_tiled ? static_cast<size_t>(kb >> 2) * 512 + (kb & 3) : static_cast<size_t>(kb);
     }
-    auto load_row = [&](int row, uint4 (&x)[2 * NCH]) {
-        const bool live = row < a.M;
-        const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(live ? row : 0) * a.ldx);
-#pragma unroll
-        for (int i = 0; i < NCH; ++i) {
-            const int kb = i * T + t;
-            const bool in = live && kb < n_blocks;
-            x[2 * i] = in ? ld_nc_16(xrow + 2 * kb) : make_uint4(0, 0, 0, 0);
-            x[2 * i + 1] = in ? ld_nc_16(xrow + 2 * kb + 1) : make_uint4(0, 0, 0, 0);
-        }
-    };
-    // four neighbouring lanes own the four blocks of one 64-channel step: one 32-bit store for their scales
-    auto store_sf = [&](int row, int kb, uint32_t sb) {
-        uint32_t word = sb << (8 * (lane & 3));
-        word |= __shfl_xor_sync(0xffffffffu, word, 1);
-        word |= __shfl_xor_sync(0xffffffffu, word, 2);
-        if ((lane & 3) == 0 && kb < n_blocks) {
-            const size_t off = sf_tiled ? nvfp4_sf_offset(row, kb, k64) : static_cast<size_t>(row) * n_blocks + kb;
-            *reinterpret_cast<uint32_t*>(sf + off) = word;
-        }
-    };
+    const bool per_token = a.clip_step == nullptr;
+    const float clip = per_token ? 0.0f : __ldg(a.clip_step);
+    const float range_max = FP4 ? kNvfp4Range : static_cast<float>(o.qmax);
+    const int k64 = a.K >> 6;
 
-    uint4 nxt[2 * NCH];
-    load_row(blockIdx.x, nxt);
-    int par = 0;
-    for (int row = blockIdx.x; row < M_pad; row += gridDim.x, par ^= 1) {
-        if (row >= a.M) {                          // padding row of the last 128-row scale atom: zero scales
+    int slot3 = 0;
+    for (int j = 0; j < n_rows; ++j) {
+        const int row = first + j * stride;
+        const size_t sf_row = !FP4 ? 0 : (o.sf_tiled ? static_cast<size_t>(row >> 7) * k64 * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4
+                                                     : static_cast<size_t>(row) * n_blocks);
+        if (j >= n_live) {                         // padding row: zero scales
+            if (FP4) {
 #pragma unroll
-            for (int i = 0; i < NCH; ++i) store_sf(row, i * T + t, 0u);
+                for (int i = 0; i < NCH; ++i)
+                    if (i * T + t < n_blocks) o.sf[sf_row + sf_col[i]] = 0;
+            }
             continue;
         }
-        float u[NCH][16];
+        const int slot = j & (kRowSlots - 1);
+        if (!mbar_wait<20>(bar0 + 8u * slot, (j / kRowSlots) & 1, &abort_word, W_ROW_FULL)) break;
+        const float g = g_slot[slot];
+        const uint32_t src = ring_addr + slot * row_bytes;
+
+        f32x2 u[NCH][8];
+        float mb[NCH];                             // per block: max |x dinv|
         float m = 0.0f;
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
-            float lo8[8], hi8[8];
-            mul_dinv8(nxt[2 * i], *reinterpret_cast<const float(*)[8]>(&dd[i][0]), lo8);
-            mul_dinv8(nxt[2 * i + 1], *reinterpret_cast<const float(*)[8]>(&dd[i][8]), hi8);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                u[i][j] = lo8[j];
-                u[i][8 + j] = hi8[j];
-                m = fmaxf(m, fmaxf(fabsf(lo8[j]), fabsf(hi8[j])));
-            }
+            const uint4 x0 = lds128(src + lds_off[i]);
+            const uint4 x1 = lds128(src + lds_off[i] + 16);
+            const float m0 = mul_dinv8(x0, &dd[i][0], &u[i][0]);
+            const float m1 = mul_dinv8(x1, &dd[i][4], &u[i][4]);
+            mb[i] = fmaxf(m0, m1);
+            m = fmaxf(m, mb[i]);
         }
-        load_row(row + gridDim.x, nxt);
-        const float g = a.gamma_step[stream_of_row(a.seg, row)];
         float range;
-        if (a.clip_step == nullptr) range = __fmul_rn(block_max(m, red[par]), g);
-        else                        range = *a.clip_step;
-        const float inv = (range != 0.0f) ? __fdiv_rn(kNvfp4Range, range) : 0.0f;
-        uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * (a.K >> 1));
+        if (per_token) range = __fmul_rn(cta_max_nonneg(m, red, slot3), g);
+        else { __syncthreads(); range = clip; }
+        // every thread has consumed the staged row: refill its slot
+        if (t == 0 && j + kRowSlots < n_live) issue(j + kRowSlots);
+        const float inv = (range != 0.0f) ? __fdiv_rn(range_max, range) : 0.0f;
+        const f32x2 g2 = pack2(g, g), inv2 = pack2(inv, inv);
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
             const int kb = i * T + t;
-            float v[16];
+            if (FP4) {
+                // The block's largest scaled magnitude is the scaled largest magnitude: both
+                // multiplications are monotonic, so no second max pass over the 16 values is needed.
+                const float vmax = __fmul_rn(__fmul_rn(mb[i], g), inv);
+                const uint32_t sb = f32_to_ue4m3(div6(vmax));
+                const float rb = rb_tab[sb];
+                const f32x2 rb2 = pack2(rb, rb);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(__fmul_rn(u[i][j], g), inv);
-            uint32_t lo, hi;
-            const uint32_t sb = nvfp4_encode_block(v, lo, hi);
-            if (kb < n_blocks) crow[kb] = make_uint2(lo, hi);
-            store_sf(row, kb, sb);
+                for (int k = 0; k < 8; ++k) { mul2(u[i][k], g2); mul2(u[i][k], inv2); mul2(u[i][k], rb2); }
+                const uint32_t lo = e2m1x8(&u[i][0]);
+                const uint32_t hi = e2m1x8(&u[i][4]);
+                if (kb < n_blocks) {
+                    *reinterpret_cast<uint2*>(static_cast<uint8_t*>(o.codes) + static_cast<size_t>(row) * o.ldc + kb * 8) = make_uint2(lo, hi);
+                    o.sf[sf_row + sf_col[i]] = static_cast<uint8_t>(sb);
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) { mul2(u[i][k], g2); mul2(u[i][k], inv2); }
+                const float qmaxf = range_max;
+                const uint2 q0 = per_token ? s8x8<false>(&u[i][0], qmaxf) : s8x8<true>(&u[i][0], qmaxf);
+                const uint2 q1 = per_token ? s8x8<false>(&u[i][4], qmaxf) : s8x8<true>(&u[i][4], qmaxf);
+                if (kb < n_blocks)
+                    *reinterpret_cast<uint4*>(static_cast<uint8_t*>(o.codes) + static_cast<size_t>(row) * o.ldc + kb * 16) = make_uint4(q0.x, q0.y, q1.x, q1.y);
+            }
         }
-        if (t == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, kNvfp4Range), g) : 0.0f;
+        if (t == 0) o.r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, range_max), g) : 0.0f;
     }
 }
 
-// Threads per CTA and pieces per thread for a row of n pieces.
-static void row_launch_shape(int n, int& threads, int& nch) {
-    nch = (n + 1023) / 1024;
+// Blocks of 16 channels per thread and threads per CTA for a row of n blocks.
+static bool row_launch_shape(int n, int& threads, int& nch) {
+    if (n > 1024) return false;
+    nch = RUDDER_ROW_NCH;
+    while (nch > 1 && n < 32 * nch) nch >>= 1;      // short rows: keep a full warp busy
     threads = ((n + nch - 1) / nch + 31) / 32 * 32;
+    return true;
 }
-static int row_grid(int rows, int threads) {
-    const int per_sm = 2048 / threads > 0 ? 2048 / threads : 1;
-    const int cap = 148 * (per_sm > 8 ? 8 : per_sm);
+// Persistent grid: as many CTAs as fit on the device at once.
+template <typename Kernel>
+static int row_grid(Kernel kernel, int rows, int threads, size_t smem) {
+    int dev = 0, sms = 148, per_sm = 1;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const int cap = sms * per_sm;
     return rows < cap ? rows : cap;
 }
 
-// The GEMMs that follow these kernels use ~200 KB of shared memory.  Asking for the same carve-out here
-// keeps the SM's L1 / shared-memory split from being reconfigured at every kernel boundary.
 cudaError_t actq_init()
 {
     cudaError_t e;
-#define RUDDER_CARVE(K)                                                                                         \
-    e = cudaFuncSetAttribute(K, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared); \
+#define RUDDER_ROW_ATTR(K)                                                                      \
+    e = cudaFuncSetAttribute(K, cudaFuncAttributeMaxDynamicSharedMemorySize, kRowSlots * 32768); \
     if (e != cudaSuccess) return e;
-    RUDDER_CARVE(actq_int_row_kernel<1>) RUDDER_CARVE(actq_int_row_kernel<2>) RUDDER_CARVE(actq_int_row_kernel<4>)
-    RUDDER_CARVE(actq_int_kernel<0>)
-    RUDDER_CARVE(actq_nvfp4_row_kernel<1>) RUDDER_CARVE(actq_nvfp4_row_kernel<2>) RUDDER_CARVE(actq_nvfp4_kernel<0>)
-#undef RUDDER_CARVE
+    RUDDER_ROW_ATTR((actq_row_kernel<true, 1>)) RUDDER_ROW_ATTR((actq_row_kernel<true, 2>)) RUDDER_ROW_ATTR((actq_row_kernel<true, 4>))
+    RUDDER_ROW_ATTR((actq_row_kernel<false, 1>)) RUDDER_ROW_ATTR((actq_row_kernel<false, 2>)) RUDDER_ROW_ATTR((actq_row_kernel<false, 4>))
+#undef RUDDER_ROW_ATTR
     return cudaSuccess;
+}
+
+// Rows can be staged by bulk copies when they start on 16-byte boundaries and are at most 16384 channels.
+template <bool FP4>
+static bool launch_row(const ActqArgs& a, const RowOut& o, int rows, cudaStream_t st)
+{
+    int threads, nch;
+    const bool aligned = (reinterpret_cast<uintptr_t>(a.X) % 16 == 0) && ((a.ldx * 2) % 16 == 0) &&
+                         (reinterpret_cast<uintptr_t>(o.codes) % 16 == 0) && (o.ldc % 16 == 0) && (a.K % 16 == 0);
+    if (!aligned || !row_launch_shape(a.K / 16, threads, nch)) return false;
+    const size_t smem = static_cast<size_t>(kRowSlots) * a.K * 2;
+    if (nch == 1)      actq_row_kernel<FP4, 1><<<row_grid(actq_row_kernel<FP4, 1>, rows, threads, smem), threads, smem, st>>>(a, o);
+    else if (nch == 2) actq_row_kernel<FP4, 2><<<row_grid(actq_row_kernel<FP4, 2>, rows, threads, smem), threads, smem, st>>>(a, o);
+    else               actq_row_kernel<FP4, 4><<<row_grid(actq_row_kernel<FP4, 4>, rows, threads, smem), threads, smem, st>>>(a, o);
+    return true;
 }
 
 cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st)
 {
     const int M_pad = sf_tiled ? ((a.M + 127) / 128) * 128 : a.M;
-    const int tiled = sf_tiled ? 1 : 0;
-    int threads, nch;
-    row_launch_shape(a.K / 16, threads, nch);
-    const int grid = row_grid(M_pad, threads);
-    if (nch == 1)      actq_nvfp4_row_kernel<1><<<grid, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
-    else if (nch == 2) actq_nvfp4_row_kernel<2><<<grid, threads, 0, st>>>(a, M_pad, codes, sf, tiled, r);
-    else {
-        const int blocks = (M_pad * 32 + 255) / 256;      // very long rows: one warp per row, row read twice
-        actq_nvfp4_kernel<0><<<blocks, 256, 0, st>>>(a, M_pad, codes, sf, tiled, r);
+    RowOut o;
+    o.codes = codes; o.ldc = a.K / 2; o.sf = sf; o.sf_tiled = sf_tiled ? 1 : 0; o.r = r; o.M_pad = M_pad; o.qmax = 0;
+    if (!launch_row<true>(a, o, M_pad, st)) {
+        const int blocks = (M_pad * 32 + 255) / 256;      // unaligned or very long rows: one warp per row, row read twice
+        actq_nvfp4_kernel<0><<<blocks, 256, 0, st>>>(a, M_pad, codes, sf, o.sf_tiled, r);
     }
     return cudaGetLastError();
 }
 
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st)
 {
-    int threads, nch;
-    row_launch_shape(a.K / 8, threads, nch);
-    const int grid = row_grid(a.M, threads);
-    if (nch == 1)      actq_int_row_kernel<1><<<grid, threads, 0, st>>>(a, qmax, codes, ldc, r);
-    else if (nch == 2) actq_int_row_kernel<2><<<grid, threads, 0, st>>>(a, qmax, codes, ldc, r);
-    else if (nch <= 4) actq_int_row_kernel<4><<<grid, threads, 0, st>>>(a, qmax, codes, ldc, r);
-    else {
-        const int blocks = (a.M * 32 + 255) / 256;         // very long rows: one warp per row, row read twice
+    RowOut o;
+    o.codes = codes; o.ldc = ldc; o.sf = nullptr; o.sf_tiled = 0; o.r = r; o.M_pad = a.M; o.qmax = qmax;
+    if (!launch_row<false>(a, o, a.M, st)) {
+        const int blocks = (a.M * 32 + 255) / 256;         // unaligned or very long rows: one warp per row, row read twice
         actq_int_kernel<0><<<blocks, 256, 0, st>>>(a, qmax, codes, ldc, r);
     }
     return cudaGetLastError();
