@@ -491,7 +491,7 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
 // Blocks of 16 channels per thread and threads per CTA for a row of n blocks.
 static bool row_launch_shape(int n, int& threads, int& nch) {
     if (n > 1024) return false;
-    nch = RUDDER_ROW_NCH;
+    nch = n > 512 ? 4 : RUDDER_ROW_NCH;             // long rows: fewer, fatter threads keep two CTAs per SM
     while (nch > 1 && n < 32 * nch) nch >>= 1;      // short rows: keep a full warp busy
     threads = ((n + nch - 1) / nch + 31) / 32 * 32;
     return true;

@@ -42,6 +42,22 @@ bool make_tmap_2d(CUtensorMap* tm, CUtensorMapDataType dt, int esize, const void
     return r == CUDA_SUCCESS;
 }
 
+// Block scales in the tensor core's order seen as [atoms][K/64][128 words of 4 bytes]; box = {128, 4, box_atoms}:
+// the four 512-byte chunks of one 256-channel stage, for box_atoms 128-row atoms.
+bool make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t k64, uint64_t atoms, uint32_t box_atoms)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t gdim[3] = {128, k64, atoms};
+    cuuint64_t gstride[2] = {512, k64 * 512};
+    cuuint32_t box[3] = {128, 4, box_atoms};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(base), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -149,7 +165,8 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
         if (launch_actq_nvfp4(a, codes4, sfx, true, r4, st) != cudaSuccess) return RUDDER_ERR_CUDA;
         if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
         GemmFp4Args g;
-        const int tt = gemm_fp4_token_tile(M);
+        const bool pair = gemm_fp4_use_pair(M, w->N, w->K);
+        const int tt = pair ? 128 : gemm_fp4_token_tile(M);
         const uint32_t box_tok = static_cast<uint32_t>(M < tt ? M : tt);
         const uint64_t kb = static_cast<uint64_t>(w->K / 2);
         if (!make_tmap_2d(&g.tm_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes4, kb, static_cast<uint64_t>(M), kb, 128, box_tok,
@@ -159,6 +176,9 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
             !make_tmap_2d(&g.tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, static_cast<uint64_t>(w->N), static_cast<uint64_t>(M),
                           static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128),
                           static_cast<uint32_t>(M < gemm_fp4_store_rows(M) ? M : gemm_fp4_store_rows(M)), CU_TENSOR_MAP_SWIZZLE_NONE))
+            return RUDDER_ERR_CUDA;
+        if (pair && (!make_tmap_sf(&g.tm_sfx, sfx, static_cast<uint64_t>(w->K / 64), static_cast<uint64_t>((M + 127) / 128), 2) ||
+                     !make_tmap_sf(&g.tm_sfw, w->sf_tiled, static_cast<uint64_t>(w->K / 64), static_cast<uint64_t>((w->N + 127) / 128), 1)))
             return RUDDER_ERR_CUDA;
         g.sm_count = sm_count();
         g.sf_x = sfx; g.sf_w = w->sf_tiled;

@@ -351,11 +351,14 @@ cudaError_t gemm_fp4_init()
 {
     cudaError_t e = cudaFuncSetAttribute(fp4::gemm_nvfp4_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, fp4::Tile<128>::DYN_SMEM);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(fp4::gemm_nvfp4_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, fp4::Tile<256>::DYN_SMEM);
+    e = cudaFuncSetAttribute(fp4::gemm_nvfp4_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, fp4::Tile<256>::DYN_SMEM);
+    if (e != cudaSuccess) return e;
+    return gemm_fp4_pair_init();
 }
 
 cudaError_t launch_gemm_fp4(const GemmFp4Args& a, cudaStream_t st)
 {
+    if (gemm_fp4_use_pair(a.M, a.N, a.K)) return launch_gemm_fp4_pair(a, st);
     return gemm_fp4_token_tile(a.M) == 256 ? launch_fp4_one<256>(a, st) : launch_fp4_one<128>(a, st);
 }
 

@@ -74,6 +74,9 @@ cudaError_t launch_pack_nvfp4(const float* W, const float* d, int N, int K, uint
 
 struct GemmFp4Args {
     CUtensorMap tm_x;           // activation codes, packed E2M1 bytes [M, K/2], box {128 bytes, token tile}, 128-byte swizzle
+                                // (CTA-pair kernel: box of 128 tokens, one half of the pair's token tile)
+    CUtensorMap tm_sfx;         // CTA-pair kernel only: activation block scales as [atoms][K/64][128 words], box {128, 4, 2}
+    CUtensorMap tm_sfw;         // CTA-pair kernel only: weight block scales, same shape, box {128, 4, 1}
     CUtensorMap tm_w;           // weight codes, packed E2M1 bytes [N, K/2], box {128 bytes, 128 channels}, 128-byte swizzle
     CUtensorMap tm_y;           // output bf16 [M, N]
     const uint8_t* sf_x;        // activation block scales, tiled [ceil(M/128)][K/64][512]
@@ -88,6 +91,9 @@ int gemm_fp4_store_rows(int M); // token rows of one TMA store box (a quarter of
 cudaError_t launch_gemm_fp4(const GemmFp4Args& a, cudaStream_t st);
 cudaError_t gemm_fp4_init();
 int gemm_fp4_token_tile(int M);
+bool gemm_fp4_use_pair(int M, int N, int K);   // two CTAs share a 256-channel x 256-token tile (cta_group::2)
+cudaError_t gemm_fp4_pair_init();
+cudaError_t launch_gemm_fp4_pair(const GemmFp4Args& a, cudaStream_t st);
 
 struct GemmI8Args {
     CUtensorMap tm_x;           // activation codes int8 [M, K], box {128 bytes, token tile}, 128-byte swizzle

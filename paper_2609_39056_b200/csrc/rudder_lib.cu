@@ -8,5 +8,6 @@
 #include "actq.cu"
 #include "gemm_i8.cu"
 #include "gemm_fp4.cu"
+#include "gemm_fp4_pair.cu"
 #include "api.cu"
 #include "static_ws.cu"
