@@ -43,7 +43,8 @@ def test_pack_export_bit_exact(rd, N, K):
 
 
 @pytest.mark.parametrize("mode", [0, 1])
-@pytest.mark.parametrize("M,K", [(1, 256), (37, 512), (130, 1024), (64, 2048), (19, 4096), (9, 8192), (5, 12288)])
+@pytest.mark.parametrize("M,K", [(1, 256), (37, 512), (130, 1024), (64, 2048), (19, 4096), (9, 8192), (5, 12288),
+                                 (300, 3072), (3, 16640)])   # many rows per CTA; rows too long to stage (warp-per-row kernel)
 def test_activation_codes_bit_exact(rd, mode, M, K):
     inp = wl.tiny(seed=500 + M, M=M, K=K, N=64, T=3)
     ref_w = oracle.pack_nvfp4(inp.W, inp.d)
@@ -68,6 +69,11 @@ CASES = [
     (300, 512, 128),       # last token tile owns a single 128-row scale atom
     (33, 2304, 256),       # 9 stages: the ring wraps
     (513, 1024, 256),
+    # M >= 1024 with whole 256-channel tiles: the CTA-pair kernel
+    (1024, 256, 256),      # one stage
+    (1100, 768, 256),      # ragged token tail (last tile owns one scale atom), fewer stages than ring slots
+    (1300, 2304, 512),     # two channel-pair tiles, the ring wraps
+    (1030, 512, 320),      # 320 channels: not whole pair tiles -> single-CTA kernel at large M
 ]
 
 
