@@ -146,8 +146,8 @@ def build_block(rd, cfg, torch, dev):
 NCU_TRAFFIC_BYTES = {
     # sum over the kernel's 4 launches of one step (profiles/gemm_nvfp4_and_actq_cfg3_metrics.md,
     # profiles/gemm_i8_w4_and_actq_cfg2_metrics.md)
-    "cfg3_nvfp4_block_h3072_f12288_m17536": 2377.7e6,
-    "cfg2_w4a8_block_h2048_f8192_m4416": 112.9e6,
+    "cfg3_nvfp4_block_h3072_f12288_m17536": 1287.4e6,
+    "cfg2_w4a8_block_h2048_f8192_m4416": 123.4e6,
 }
 
 
@@ -216,7 +216,7 @@ def roofline_of(cfg, m, pk):
     else:
         pro_bytes = sum(2 * M * K + M * K + 4 * M for _, K, N in cfg.linears)
     traffic = NCU_TRAFFIC_BYTES.get(cfg.name)
-    return {"kernel": "gemm_nvfp4_kernel" if cfg.scheme == "nvfp4" else "gemm_i8_w4_kernel", "launches_per_step": 4,
+    return {"kernel": "gemm_nvfp4_pair_kernel" if cfg.scheme == "nvfp4" else "gemm_i8_w4_kernel", "launches_per_step": 4,
             "bound": "tensor", "achieved": achieved, "peak": tensor_peak,
             "unit": "TFLOP/s" if cfg.scheme == "nvfp4" else "TOPS", "frac": achieved / tensor_peak,
             "peak_source": f"{pk['source']} bf16 sustained {pk['bf16_sustained']} x {ratio:g} (nominal ratio), of measured",

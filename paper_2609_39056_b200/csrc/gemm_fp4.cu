@@ -68,8 +68,10 @@ struct Params {
 
 enum Where { W_EMPTY = 601, W_FULL = 701, W_ACC_EMPTY = 702, W_ACC_FULL = 801 };
 
+// No memory clobber: the loads of the token scales may move across these stores; the fence and
+// barrier that follow are volatile too and keep their place relative to the stores.
 __device__ __forceinline__ void sts16(uint32_t addr, uint16_t v) {
-    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v));
 }
 // 1D bulk copy global -> shared, completion counted on an mbarrier (addresses and size multiples of 16).
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {

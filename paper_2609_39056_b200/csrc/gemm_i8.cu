@@ -140,8 +140,11 @@ enum Where {   // codes recorded when a bounded wait gives up
 __device__ __forceinline__ void sts128(uint32_t addr, const uint4& v) {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
+// No memory clobber: the compiler may move the loads of the token scales across these stores (with a
+// clobber every store waits for the load before it); the fence and barrier that follow are volatile
+// too and keep their place relative to the stores.
 __device__ __forceinline__ void sts16(uint32_t addr, uint16_t v) {
-    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v));
 }
 __device__ __forceinline__ uint4 ldg_nc_16(const void* p) {
     uint4 v;
