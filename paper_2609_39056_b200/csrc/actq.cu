@@ -59,6 +59,7 @@ template <int NIT>
 __global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int8_t* __restrict__ codes, int64_t ldc,
                                                         float* __restrict__ r)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // may have been launched ahead of its stream predecessors
     const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (row >= a.M) return;
@@ -150,6 +151,7 @@ template <int NIT>
 __global__ void __launch_bounds__(256) actq_nvfp4_kernel(ActqArgs a, int M_pad, uint8_t* __restrict__ codes,
                                                           uint8_t* __restrict__ sf, int sf_tiled, float* __restrict__ r)
 {
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // may have been launched ahead of its stream predecessors
     const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (row >= M_pad) return;
@@ -368,8 +370,6 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
     // Let a dependent GEMM launched with programmatic dependent launch start its own set-up now; it
     // still waits for this whole grid to finish before it reads anything written here.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (blockIdx.x == 0 && a.zero_ints != nullptr)
-        for (int i = t; i < a.n_zero; i += T) a.zero_ints[i] = 0;
     if (t == 0) {
         abort_word = 0;
         for (int i = 0; i < kRowSlots; ++i) mbar_init(bar0 + 8u * i, 1);
@@ -389,16 +389,6 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
     const int M_rows = FP4 ? o.M_pad : M;
     const int n_rows = first < M_rows ? (M_rows - 1 - first) / stride + 1 : 0;
     const int n_live = first < M ? (M - 1 - first) / stride + 1 : 0;
-    auto issue = [&](int j) {                                  // thread 0: stage row j of this CTA
-        const int slot = j & (kRowSlots - 1);
-        const int row = first + j * stride;
-        g_slot[slot] = __ldg(a.gamma_step + stream_of_row(a.seg, row));
-        mbar_expect_tx(bar0 + 8u * slot, row_bytes);
-        bulk_row_load(ring_addr + slot * row_bytes, a.X + static_cast<size_t>(row) * a.ldx, row_bytes, bar0 + 8u * slot);
-    };
-    if (t == 0)
-        for (int j = 0; j < kRowSlots && j < n_live; ++j) issue(j);
-
     f32x2 dd[NCH][8];
     uint32_t lds_off[NCH];                         // byte offset of the thread's blocks in a staged row
     size_t sf_col[NCH];                            // column part of the scale's address
@@ -414,6 +404,22 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
         lds_off[i] = static_cast<uint32_t>(kb < n_blocks ? kb : n_blocks - 1) * 32u;   // spare threads re-read the last block (their dinv is 0)
         sf_col[i] = o.sf_tiled ? static_cast<size_t>(kb >> 2) * 512 + (kb & 3) : static_cast<size_t>(kb);
     }
+    // This kernel may itself have been launched early (programmatic dependent launch): everything above
+    // touches only what belongs to the weights or to this CTA.  From here on it reads X and writes the
+    // workspace, which the kernels before it in the stream may still be producing or reading.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (blockIdx.x == 0 && a.zero_ints != nullptr)
+        for (int i = t; i < a.n_zero; i += T) a.zero_ints[i] = 0;
+    auto issue = [&](int j) {                                  // thread 0: stage row j of this CTA
+        const int slot = j & (kRowSlots - 1);
+        const int row = first + j * stride;
+        g_slot[slot] = __ldg(a.gamma_step + stream_of_row(a.seg, row));
+        mbar_expect_tx(bar0 + 8u * slot, row_bytes);
+        bulk_row_load(ring_addr + slot * row_bytes, a.X + static_cast<size_t>(row) * a.ldx, row_bytes, bar0 + 8u * slot);
+    };
+    if (t == 0)
+        for (int j = 0; j < kRowSlots && j < n_live; ++j) issue(j);
+
     const bool per_token = a.clip_step == nullptr;
     const float clip = per_token ? 0.0f : __ldg(a.clip_step);
     const float range_max = FP4 ? kNvfp4Range : static_cast<float>(o.qmax);
@@ -488,6 +494,28 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
     }
 }
 
+// Launch that may start before the kernels ahead of it in the stream have finished (programmatic
+// dependent launch); the kernel itself waits (griddepcontrol.wait) before it touches their data.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_early(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+#ifdef RUDDER_DBG_NO_K1PDL
+    cfg.numAttrs = 0;
+#else
+    cfg.numAttrs = 1;
+#endif
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // Blocks of 16 channels per thread and threads per CTA for a row of n blocks.
 static bool row_launch_shape(int n, int& threads, int& nch) {
     if (n > 1024) return false;
@@ -521,16 +549,16 @@ cudaError_t actq_init()
 
 // Rows can be staged by bulk copies when they start on 16-byte boundaries and are at most 16384 channels.
 template <bool FP4>
-static bool launch_row(const ActqArgs& a, const RowOut& o, int rows, cudaStream_t st)
+static bool launch_row(const ActqArgs& a, const RowOut& o, int rows, cudaStream_t st, cudaError_t* err)
 {
     int threads, nch;
     const bool aligned = (reinterpret_cast<uintptr_t>(a.X) % 16 == 0) && ((a.ldx * 2) % 16 == 0) &&
                          (reinterpret_cast<uintptr_t>(o.codes) % 16 == 0) && (o.ldc % 16 == 0) && (a.K % 16 == 0);
     if (!aligned || !row_launch_shape(a.K / 16, threads, nch)) return false;
     const size_t smem = static_cast<size_t>(kRowSlots) * a.K * 2;
-    if (nch == 1)      actq_row_kernel<FP4, 1><<<row_grid(actq_row_kernel<FP4, 1>, rows, threads, smem), threads, smem, st>>>(a, o);
-    else if (nch == 2) actq_row_kernel<FP4, 2><<<row_grid(actq_row_kernel<FP4, 2>, rows, threads, smem), threads, smem, st>>>(a, o);
-    else               actq_row_kernel<FP4, 4><<<row_grid(actq_row_kernel<FP4, 4>, rows, threads, smem), threads, smem, st>>>(a, o);
+    if (nch == 1)      *err = launch_early(actq_row_kernel<FP4, 1>, row_grid(actq_row_kernel<FP4, 1>, rows, threads, smem), threads, smem, st, a, o);
+    else if (nch == 2) *err = launch_early(actq_row_kernel<FP4, 2>, row_grid(actq_row_kernel<FP4, 2>, rows, threads, smem), threads, smem, st, a, o);
+    else               *err = launch_early(actq_row_kernel<FP4, 4>, row_grid(actq_row_kernel<FP4, 4>, rows, threads, smem), threads, smem, st, a, o);
     return true;
 }
 
@@ -539,22 +567,25 @@ cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bo
     const int M_pad = sf_tiled ? ((a.M + 127) / 128) * 128 : a.M;
     RowOut o;
     o.codes = codes; o.ldc = a.K / 2; o.sf = sf; o.sf_tiled = sf_tiled ? 1 : 0; o.r = r; o.M_pad = M_pad; o.qmax = 0;
-    if (!launch_row<true>(a, o, M_pad, st)) {
+    cudaError_t err = cudaSuccess;
+    if (!launch_row<true>(a, o, M_pad, st, &err)) {
         const int blocks = (M_pad * 32 + 255) / 256;      // unaligned or very long rows: one warp per row, row read twice
-        actq_nvfp4_kernel<0><<<blocks, 256, 0, st>>>(a, M_pad, codes, sf, o.sf_tiled, r);
+        err = launch_early(actq_nvfp4_kernel<0>, blocks, 256, 0, st, a, M_pad, codes, sf, o.sf_tiled, r);
     }
-    return cudaGetLastError();
+    return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st)
 {
     RowOut o;
     o.codes = codes; o.ldc = ldc; o.sf = nullptr; o.sf_tiled = 0; o.r = r; o.M_pad = a.M; o.qmax = qmax;
-    if (!launch_row<false>(a, o, a.M, st)) {
+    cudaError_t err = cudaSuccess;
+    if (!launch_row<false>(a, o, a.M, st, &err)) {
         const int blocks = (a.M * 32 + 255) / 256;         // unaligned or very long rows: one warp per row, row read twice
-        actq_int_kernel<0><<<blocks, 256, 0, st>>>(a, qmax, codes, ldc, r);
+        if (a.zero_ints != nullptr && cudaMemsetAsync(a.zero_ints, 0, sizeof(int) * a.n_zero, st) != cudaSuccess) return cudaErrorUnknown;
+        err = launch_early(actq_int_kernel<0>, blocks, 256, 0, st, a, qmax, codes, ldc, r);
     }
-    return cudaGetLastError();
+    return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace rudder

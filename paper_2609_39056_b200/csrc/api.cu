@@ -216,6 +216,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
                       CU_TENSOR_MAP_SWIZZLE_NONE))
         return RUDDER_ERR_CUDA;
     g.w_codes = w->codes; g.w_scales_t = w->scales_t;
+    g.y = Y; g.ldy = ldy;
     g.M = M; g.N = w->N; g.K = w->K; g.G = w->G;
     g.row_scale = r; g.bias = bias;
     g.acc = acc; g.row0 = row0; g.rows = rows; g.col0 = col0; g.cols = cols;

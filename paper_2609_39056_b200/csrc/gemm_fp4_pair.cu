@@ -162,6 +162,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_word;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the next prologue kernel may start its own set-up
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)

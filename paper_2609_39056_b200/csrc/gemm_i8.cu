@@ -105,12 +105,16 @@ struct Params {
     const float* scales_t;       // [K/G][N] fp32 = Delta_W / 16
     const float* row_scale;      // r [M]
     const float* bias;           // [N] or nullptr
-    int32_t* acc;                // accumulator dump [K/G][rows][cols] or nullptr
-    int row0, rows, col0, cols;
+    // The parity hook's window and the plain output pointer share storage (a launch uses one of them):
+    // kernel parameters beyond 376 bytes cost this kernel 7 % at large M, measured.
+    union {
+        struct { int32_t* acc; int row0, rows, col0, cols; } dump;    // accumulator dump [K/G][rows][cols]
+        struct { uint16_t* y; int64_t ldy; } out;                     // output bf16 [M, ldy]: tiles of 32 / 64 tokens are stored without TMA
+    } aux;
     int m_tiles, n_tiles;        // token tiles, channel tiles (grid.x = m_tiles * n_tiles)
     int splitk;                  // K splits (grid.y)
     int stages_per_split;        // 128-channel stages per split
-    float* partials;             // [splitk][N][m_tiles * TT] fp32 partial sums (splitk > 1)
+    float* partials;             // [splitk][m_tiles * TT][N] fp32 partial sums (splitk > 1)
     int* counters;               // [m_tiles * n_tiles] arrivals per tile, zeroed by the prologue kernel
     int pdl;                     // launched with programmatic dependent launch
     uint32_t x_tx;               // bytes one activation TMA box delivers
@@ -160,6 +164,11 @@ __device__ __forceinline__ float ldg_f32_volatile(const float* p) {
 __device__ __forceinline__ float ld_f32_volatile(const float* p) {
     float v;
     asm volatile("ld.global.f32 %0, [%1];" : "=f"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ float ld_f32_cg(const float* p) {     // from L2; no clobber, so that several can be in flight
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
     return v;
 }
 __device__ __forceinline__ float4 ld_f32x4_volatile(const float* p) {
@@ -224,6 +233,9 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_word;
+#ifndef RUDDER_DBG_NO_TRIGGER
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the next prologue kernel may start its own set-up
+#endif
 
     if (warp < 8) {
     // The epilogue warpgroups hold TT/2 fp32 accumulators per thread: hand them the registers the
@@ -520,14 +532,14 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     acc[ch * CH + j] = fmaf(__int2float_rn(static_cast<int>(cur[j])), sc, acc[ch * CH + j]);
 #endif
                 if (DUMP) {
-                    const int cc = n - p.col0;
-                    if (p.acc != nullptr && n_ok && cc >= 0 && cc < p.cols) {
+                    const int cc = n - p.aux.dump.col0;
+                    if (p.aux.dump.acc != nullptr && n_ok && cc >= 0 && cc < p.aux.dump.cols) {
 #pragma unroll
                         for (int j = 0; j < CH; ++j) {
                             const int tok = m0 + h * EC + ch * CH + j;
-                            const int rr = tok - p.row0;
-                            if (tok < p.M && rr >= 0 && rr < p.rows)
-                                p.acc[(static_cast<size_t>(g0 + g) * p.rows + rr) * p.cols + cc] = static_cast<int>(cur[j]) >> 4;
+                            const int rr = tok - p.aux.dump.row0;
+                            if (tok < p.M && rr >= 0 && rr < p.aux.dump.rows)
+                                p.aux.dump.acc[(static_cast<size_t>(g0 + g) * p.aux.dump.rows + rr) * p.aux.dump.cols + cc] = static_cast<int>(cur[j]) >> 4;
                         }
                     }
                 }
@@ -547,30 +559,49 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // Split K: publish this split's partial sums; the CTA that arrives last at the tile's counter adds
         // the splits in order and goes on to write the tile, the others are done.
         bool writer = true;
-        if (TT <= 128 && p.splitk > 1) {           // only small-M launches split K
+        if (TT <= 64 && p.splitk > 1) {            // only launches with tiles of 32 / 64 tokens split K
             const int m_pad = p.m_tiles * TT;
-            float* mine = p.partials + (static_cast<size_t>(blockIdx.y) * p.N + (n_ok ? n : 0)) * m_pad + m0 + h * EC;
+            // partials[split][token][channel]: a warp (32 consecutive channels) writes and reads whole
+            // 128-byte lines.  (With the channel outermost every lane touched its own line, and the
+            // reduction spent its time in the L1 tag stage: 32 lines per load instruction.)
+            float* mine = p.partials + (static_cast<size_t>(blockIdx.y) * m_pad + m0 + h * EC) * p.N + (n_ok ? n : 0);
             if (ok && n_ok) {
 #pragma unroll
-                for (int j = 0; j < EC; j += 4)
-                    *reinterpret_cast<float4*>(mine + j) = make_float4(acc[j], acc[j + 1], acc[j + 2], acc[j + 3]);
+                for (int j = 0; j < EC; ++j) mine[static_cast<size_t>(j) * p.N] = acc[j];
             }
-            __threadfence();
+            // The barrier orders every drain thread's stores before thread 256's release; its acquire on
+            // the other side, again followed by a barrier, orders them before the readers' loads (which
+            // go to L2).  One round trip instead of a fence per thread plus an atomic.
             asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
-            if (threadIdx.x == 256) last_flag = (atomicAdd(p.counters + blockIdx.x, 1) == p.splitk - 1) ? 1 : 0;
+            if (threadIdx.x == 256) {
+                int old;
+                asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(p.counters + blockIdx.x) : "memory");
+                last_flag = (old == p.splitk - 1) ? 1 : 0;
+            }
             asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
             writer = last_flag != 0;
             if (writer && ok) {
-                __threadfence();
 #pragma unroll
                 for (int j = 0; j < EC; ++j) acc[j] = 0.0f;
                 if (n_ok) {
-                    for (int z = 0; z < p.splitk; ++z) {
-                        const float* src = p.partials + (static_cast<size_t>(z) * p.N + n) * m_pad + m0 + h * EC;
+                    // ZB splits are requested together (the loads of one split alone would expose one L2
+                    // round trip per split) and added in split order.
+                    constexpr int ZB = (EC >= 64) ? 1 : 64 / EC;
+                    for (int z0 = 0; z0 < p.splitk; z0 += ZB) {
+                        float v[ZB][EC];
 #pragma unroll
-                        for (int j = 0; j < EC; j += 4) {
-                            const float4 v = ld_f32x4_volatile(src + j);
-                            acc[j] += v.x; acc[j + 1] += v.y; acc[j + 2] += v.z; acc[j + 3] += v.w;
+                        for (int zz = 0; zz < ZB; ++zz) {
+                            const int z = (z0 + zz < p.splitk) ? z0 + zz : p.splitk - 1;
+                            const float* src = p.partials + (static_cast<size_t>(z) * m_pad + m0 + h * EC) * p.N + n;
+#pragma unroll
+                            for (int j = 0; j < EC; ++j) v[zz][j] = ld_f32_cg(src + static_cast<size_t>(j) * p.N);
+                        }
+#pragma unroll
+                        for (int zz = 0; zz < ZB; ++zz) {
+                            if (z0 + zz < p.splitk) {
+#pragma unroll
+                                for (int j = 0; j < EC; ++j) acc[j] += v[zz][j];
+                            }
                         }
                     }
                 }
@@ -580,6 +611,20 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // stage the transposed bf16 tile there ([token][channel], `out_pitch` channels per row).
         ok = ok && writer;
         if (ok) ok = mbar_wait<64>(rs_full, 0, abortp, W_RS_FULL);
+        if (TT <= 64 && !DUMP) {
+            // Small tiles: 16 or 32 results per thread go straight to global memory (a warp writes 64
+            // contiguous bytes per token); nothing to stage, no store to wait for.
+            if (ok && n_ok) {
+                const float b = (p.bias != nullptr) ? __ldg(p.bias + n) : 0.0f;
+                uint16_t* yp = p.aux.out.y + static_cast<size_t>(m0 + h * EC) * p.aux.out.ldy + n;
+#pragma unroll
+                for (int j = 0; j < EC; ++j) {
+                    if (m0 + h * EC + j < p.M)
+                        yp[static_cast<size_t>(j) * p.aux.out.ldy] = __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j], rs_smem[h * EC + j], b)));
+                }
+            }
+            ok = false;                                          // nothing left for the staged path below
+        }
         if (ok) {
             const float b = (p.bias != nullptr && n_ok) ? __ldg(p.bias + n) : 0.0f;
             const uint32_t stage0 = smem_base + T::OFF_X;
@@ -631,13 +676,10 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.G;
     p.codes = a.w_codes; p.scales_t = a.w_scales_t;
     p.row_scale = a.row_scale; p.bias = a.bias;
-    p.acc = a.acc; p.row0 = a.row0; p.rows = a.rows; p.col0 = a.col0; p.cols = a.cols;
+    if (DUMP) { p.aux.dump.acc = a.acc; p.aux.dump.row0 = a.row0; p.aux.dump.rows = a.rows; p.aux.dump.col0 = a.col0; p.aux.dump.cols = a.cols; }
+    else      { p.aux.out.y = a.y; p.aux.out.ldy = a.ldy; }
     p.x_tx = static_cast<uint32_t>(min(TT, a.M)) * KSTAGE;
     p.out_pitch = min(BN, a.N);
-#ifdef RUDDER_ROLE_PROF
-    p.prof = reinterpret_cast<long long*>(a.acc);   // development build only: the dump pointer carries the counters
-    p.acc = nullptr;
-#endif
     p.m_tiles = (a.M + TT - 1) / TT;
     p.n_tiles = (a.N + BN - 1) / BN;
     p.splitk = plan.splitk;
@@ -666,7 +708,7 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
 GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump)
 {
     GemmI8Plan plan;
-    plan.token_tile = M > 128 ? 256 : (M > 64 ? 128 : (M > 32 ? 64 : 32));
+    plan.token_tile = M > 128 ? 256 : (M > 32 ? 64 : 32);
     plan.splitk = 1;
     plan.pdl = false;
 #ifdef RUDDER_ROLE_PROF
@@ -679,6 +721,7 @@ GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump)
     const int base = m_tiles * n_tiles;
     const size_t m_pad = static_cast<size_t>(m_tiles) * plan.token_tile;
     int sk = 1;
+    if (plan.token_tile > 64) { plan.pdl = true; return plan; }     // K is split for tiles of 32 / 64 tokens only
     while (sk < 16 && base * (sk * 2) <= 160 && (K / KSTAGE) % (sk * 2) == 0 && K / (sk * 2) >= 2 * KSTAGE &&
            static_cast<size_t>(sk * 2) * N * m_pad * sizeof(float) <= (size_t(2) << 20))
         sk *= 2;

@@ -98,6 +98,8 @@ cudaError_t launch_gemm_fp4_pair(const GemmFp4Args& a, cudaStream_t st);
 struct GemmI8Args {
     CUtensorMap tm_x;           // activation codes int8 [M, K], box {128 bytes, token tile}, 128-byte swizzle
     CUtensorMap tm_y;           // output bf16 [M, N] (row pitch ldy), box {min(128, N) channels, token tile}
+    uint16_t* y;                // the same output as a plain pointer (small tiles are stored without TMA)
+    int64_t ldy;
     const uint8_t* w_codes;     // packed INT4 weights
     const float* w_scales_t;    // [K/G][N]
     int M, N, K, G;
