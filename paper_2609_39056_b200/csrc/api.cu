@@ -166,7 +166,8 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
         if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
         GemmFp4Args g;
         const bool pair = gemm_fp4_use_pair(M, w->N, w->K);
-        const int tt = pair ? 128 : gemm_fp4_token_tile(M);
+        const int tt = pair ? 128 : gemm_fp4_token_tile(M, w->N);      // token rows of one activation box
+        const int st_rows = pair ? 64 : gemm_fp4_store_rows(M, w->N);  // token rows of one output store box
         const uint32_t box_tok = static_cast<uint32_t>(M < tt ? M : tt);
         const uint64_t kb = static_cast<uint64_t>(w->K / 2);
         if (!make_tmap_2d(&g.tm_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, codes4, kb, static_cast<uint64_t>(M), kb, 128, box_tok,
@@ -175,7 +176,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
                           static_cast<uint32_t>(w->N < 128 ? w->N : 128), CU_TENSOR_MAP_SWIZZLE_128B) ||
             !make_tmap_2d(&g.tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, static_cast<uint64_t>(w->N), static_cast<uint64_t>(M),
                           static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128),
-                          static_cast<uint32_t>(M < gemm_fp4_store_rows(M) ? M : gemm_fp4_store_rows(M)), CU_TENSOR_MAP_SWIZZLE_NONE))
+                          static_cast<uint32_t>(M < st_rows ? M : st_rows), CU_TENSOR_MAP_SWIZZLE_NONE))
             return RUDDER_ERR_CUDA;
         if (pair && (!make_tmap_sf(&g.tm_sfx, sfx, static_cast<uint64_t>(w->K / 64), static_cast<uint64_t>((M + 127) / 128), 2) ||
                      !make_tmap_sf(&g.tm_sfw, w->sf_tiled, static_cast<uint64_t>(w->K / 64), static_cast<uint64_t>((w->N + 127) / 128), 1)))

@@ -22,6 +22,8 @@
 
 namespace rudder {
 
+constexpr int BN_FP4 = 128;        // output channels per single-CTA tile
+
 namespace fp4 {
 
 constexpr int BN = 128;            // output channels per tile (MMA M)
@@ -347,8 +349,14 @@ static cudaError_t launch_fp4_one(const GemmFp4Args& a, cudaStream_t st)
     return cudaGetLastError();
 }
 
-int gemm_fp4_token_tile(int M) { return M > 128 ? 256 : 128; }
-int gemm_fp4_store_rows(int M) { return gemm_fp4_token_tile(M) / 4; }
+// 256-token tiles once they fill the device; smaller problems get twice the CTAs from 128-token tiles.
+int gemm_fp4_token_tile(int M, int N)
+{
+    if (M <= 128) return 128;
+    const long long tiles256 = static_cast<long long>((M + 255) / 256) * ((N + BN_FP4 - 1) / BN_FP4);
+    return tiles256 >= 148 ? 256 : 128;
+}
+int gemm_fp4_store_rows(int M, int N) { return gemm_fp4_token_tile(M, N) / 4; }
 
 cudaError_t gemm_fp4_init()
 {
@@ -362,7 +370,7 @@ cudaError_t gemm_fp4_init()
 cudaError_t launch_gemm_fp4(const GemmFp4Args& a, cudaStream_t st)
 {
     if (gemm_fp4_use_pair(a.M, a.N, a.K)) return launch_gemm_fp4_pair(a, st);
-    return gemm_fp4_token_tile(a.M) == 256 ? launch_fp4_one<256>(a, st) : launch_fp4_one<128>(a, st);
+    return gemm_fp4_token_tile(a.M, a.N) == 256 ? launch_fp4_one<256>(a, st) : launch_fp4_one<128>(a, st);
 }
 
 }  // namespace rudder

@@ -87,10 +87,10 @@ struct GemmFp4Args {
     const float* bias;
     int sm_count;               // persistent grid size
 };
-int gemm_fp4_store_rows(int M); // token rows of one TMA store box (a quarter of the token tile)
+int gemm_fp4_store_rows(int M, int N); // token rows of one TMA store box of the single-CTA kernel (a quarter of its token tile)
 cudaError_t launch_gemm_fp4(const GemmFp4Args& a, cudaStream_t st);
 cudaError_t gemm_fp4_init();
-int gemm_fp4_token_tile(int M);
+int gemm_fp4_token_tile(int M, int N);
 bool gemm_fp4_use_pair(int M, int N, int K);   // two CTAs share a 256-channel x 256-token tile (cta_group::2)
 cudaError_t gemm_fp4_pair_init();
 cudaError_t launch_gemm_fp4_pair(const GemmFp4Args& a, cudaStream_t st);
