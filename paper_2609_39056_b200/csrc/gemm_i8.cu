@@ -119,20 +119,8 @@ struct Params {
     int pdl;                     // launched with programmatic dependent launch
     uint32_t x_tx;               // bytes one activation TMA box delivers
     int out_pitch;               // channels per row of the staged output tile (= TMA store box width)
-#ifdef RUDDER_ROLE_PROF
-    long long* prof;             // [16] cycle counters of CTA (0,0): where each role waits (development aid)
-#endif
 };
 
-#ifdef RUDDER_ROLE_PROF
-#define PROF_DECL(n) long long prof_##n = 0
-#define PROF_WAIT(n, expr) [&]() { const long long t_ = clock64(); const bool r_ = (expr); prof_##n += clock64() - t_; return r_; }()
-#define PROF_PUT(i, n) do { if (blockIdx.x == 0 && blockIdx.y == 0 && p.prof) p.prof[i] = prof_##n; } while (0)
-#else
-#define PROF_DECL(n)
-#define PROF_WAIT(n, expr) (expr)
-#define PROF_PUT(i, n)
-#endif
 
 enum Where {   // codes recorded when a bounded wait gives up
     W_X_EMPTY = 101,
@@ -249,18 +237,16 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             if (p.pdl) griddep_wait();                 // the activation codes come from the prologue kernel
             int issued = 0;
             bool ok = true;
-            PROF_DECL(x_empty);
             int slot = 0;
             uint32_t ph = 0;
             for (int s = 0; s < n_stages; ++s) {
-                ok = PROF_WAIT(x_empty, mbar_wait<RUDDER_SLEEP_PROD>(x_empty(slot), ph ^ 1u, abortp, W_X_EMPTY));
+                ok = mbar_wait<RUDDER_SLEEP_PROD>(x_empty(slot), ph ^ 1u, abortp, W_X_EMPTY);
                 if (!ok) break;
                 mbar_expect_tx(x_full(slot), p.x_tx);
                 tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, (s0 + s) * KSTAGE, m0, x_full(slot));
                 ++issued;
                 if (++slot == T::SX) { slot = 0; ph ^= 1u; }
             }
-            PROF_PUT(0, x_empty);
             if (!ok) {
                 // Gave up: let the copies already in flight land before the CTA's shared memory goes away.
                 for (int i = max(0, issued - T::SX); i < issued; ++i)
@@ -275,10 +261,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             const bool leader = elect_one();
             const uint32_t idesc = umma_idesc_i8(BN, TT);
             bool ok = true;
-            PROF_DECL(x_full); PROF_DECL(w_full); PROF_DECL(acc_empty); PROF_DECL(mma_total);
-#ifdef RUDDER_ROLE_PROF
-            const long long mma_t0 = clock64();
-#endif
             // No divisions in this loop: every instruction on this path is latency the tensor core may
             // end up waiting for.
             const int mma_per_group = g_len >> 5;      // MMAs (K = 32 each) per weight group
@@ -288,8 +270,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             int sx = 0, sw = 0;                        // ring slots
             uint32_t phx = 0, phw = 0;                 // ring phases
             for (int s = 0; s < n_stages && ok; ++s) {
-                ok = PROF_WAIT(x_full, mbar_wait<RUDDER_SLEEP_MMA>(x_full(sx), phx, abortp, W_X_FULL)) &&
-                     PROF_WAIT(w_full, mbar_wait<RUDDER_SLEEP_MMA>(w_full(sw), phw, abortp, W_W_FULL));
+                ok = mbar_wait<RUDDER_SLEEP_MMA>(x_full(sx), phx, abortp, W_X_FULL) &&
+                     mbar_wait<RUDDER_SLEEP_MMA>(w_full(sw), phw, abortp, W_W_FULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tcgen05_fence_after_sync();
@@ -298,7 +280,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
                 for (int kk = 0; kk < KSTAGE / 32; ++kk) {
                     if (in_group == 0 && g_issued >= T::NBUF) {     // a buffer's first use needs no wait
-                        ok = PROF_WAIT(acc_empty, mbar_wait<RUDDER_SLEEP_MMA>(acc_empty(buf), phb ^ 1u, abortp, W_ACC_EMPTY));
+                        ok = mbar_wait<RUDDER_SLEEP_MMA>(acc_empty(buf), phb ^ 1u, abortp, W_ACC_EMPTY);
                         ok = __all_sync(0xffffffffu, ok);
                         if (!ok) break;
                         tcgen05_fence_after_sync();
@@ -320,10 +302,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 if (++sx == T::SX) { sx = 0; phx ^= 1u; }
                 if (++sw == SW) { sw = 0; phw ^= 1u; }
             }
-#ifdef RUDDER_ROLE_PROF
-            prof_mma_total = clock64() - mma_t0;
-#endif
-            if (leader) { PROF_PUT(3, x_full); PROF_PUT(4, w_full); PROF_PUT(5, acc_empty); PROF_PUT(6, mma_total); }
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ row scales of the tile -> shared
@@ -336,10 +314,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // 128 channels x 64 packed bytes per stage = 512 16-byte pieces, 4 per thread: piece idx covers
         // channel idx / 4, input channels [32 (idx % 4), 32 (idx % 4) + 32) of the stage.
         const int tid = threadIdx.x - 128;
-        PROF_DECL(w_empty); PROF_DECL(unpack_total);
-#ifdef RUDDER_ROLE_PROF
-        const long long un_t0 = clock64();
-#endif
         const size_t row_bytes = static_cast<size_t>(p.K / 2);
         const uint8_t* src[4];
         bool valid[4];
@@ -374,7 +348,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
                     for (int i = 0; i < 4; ++i) cur[i] = pre[j][i];
                     if (s + PD < n_stages) load_stage(s + PD, pre[j]);
-                    ok = PROF_WAIT(w_empty, mbar_wait<RUDDER_SLEEP_UNPACK>(w_empty(sw), phw ^ 1u, abortp, W_W_EMPTY));
+                    ok = mbar_wait<RUDDER_SLEEP_UNPACK>(w_empty(sw), phw ^ 1u, abortp, W_W_EMPTY);
                     if (ok) {
                         const uint32_t dst = smem_base + T::OFF_W + sw * W_BYTES;
 #pragma unroll
@@ -399,10 +373,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 }
             }
         }
-#ifdef RUDDER_ROLE_PROF
-        prof_unpack_total = clock64() - un_t0;
-        if (tid == 0) { PROF_PUT(8, w_empty); PROF_PUT(9, unpack_total); }
-#endif
     }
     } else {
         // ------------------------------------------------------------------ epilogue
@@ -419,10 +389,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
         for (int j = 0; j < EC; ++j) acc[j] = 0.0f;
         bool ok = true;
-        PROF_DECL(acc_full); PROF_DECL(epi_total); PROF_DECL(epi_drain); PROF_DECL(epi_tail); PROF_DECL(epi_vote); PROF_DECL(epi_fence);
-#ifdef RUDDER_ROLE_PROF
-        const long long ep_t0 = clock64();
-#endif
         // Scales are fetched two groups ahead with volatile loads: a plain load would be sunk next to
         // its use and expose the L2 latency once per group.
         const float* sc_ptr = p.scales_t + static_cast<size_t>(g0) * p.N + (n_ok ? n : 0);
@@ -481,23 +447,10 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             if (g + 2 < n_groups) sc_next2 = ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + 2) * p.N);
             // lane 0 polls, the others wait at the shuffle: no 32-way spin, and the verdict is warp-uniform
             // (the TMEM loads below are warp-collective)
-            if (lane == 0) ok = PROF_WAIT(acc_full, mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), phb, abortp, W_ACC_FULL));
-#ifdef RUDDER_ROLE_PROF
-            const long long v_t0 = clock64();
-#endif
+            if (lane == 0) ok = mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), phb, abortp, W_ACC_FULL);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-#ifdef RUDDER_ROLE_PROF
-            const long long f_t0 = clock64();
-            prof_epi_vote += f_t0 - v_t0;
-#endif
             tcgen05_fence_after_sync();
-#ifdef RUDDER_ROLE_PROF
-            prof_epi_fence += clock64() - f_t0;
-#endif
-#ifdef RUDDER_ROLE_PROF
-            const long long dr_t0 = clock64();
-#endif
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * TT + h * EC;
             uint32_t c0[CH], c1[CH];
 #if RUDDER_EPI_DB
@@ -548,14 +501,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(buf));  // one arrival per warp: arrivals on one barrier serialise
             if (++buf == T::NBUF) { buf = 0; phb ^= 1u; }
-#ifdef RUDDER_ROLE_PROF
-            prof_epi_drain += clock64() - dr_t0;
-#endif
         }
-#ifdef RUDDER_ROLE_PROF
-        prof_epi_total = clock64() - ep_t0;
-        const long long tail_t0 = clock64();
-#endif
         // Split K: publish this split's partial sums; the CTA that arrives last at the tile's counter adds
         // the splits in order and goes on to write the tile, the others are done.
         bool writer = true;
@@ -650,10 +596,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         }
-#ifdef RUDDER_ROLE_PROF
-        prof_epi_tail = clock64() - tail_t0;
-        if (threadIdx.x == 256) { PROF_PUT(10, epi_drain); PROF_PUT(11, acc_full); PROF_PUT(12, epi_total); PROF_PUT(13, epi_tail); PROF_PUT(14, epi_vote); PROF_PUT(15, epi_fence); }
-#endif
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -711,9 +653,6 @@ GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump)
     plan.token_tile = M > 128 ? 256 : (M > 32 ? 64 : 32);
     plan.splitk = 1;
     plan.pdl = false;
-#ifdef RUDDER_ROLE_PROF
-    dump = false;               // development build: the dump pointer carries cycle counters, not accumulators
-#endif
     if (dump || M > 256) return plan;
     const int n_tiles = (N + BN - 1) / BN;
     if (M > 128 && n_tiles < 74) plan.token_tile = 128;       // two token tiles double the CTAs
@@ -758,11 +697,7 @@ cudaError_t gemm_i8_init()
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st)
 {
     const GemmI8Plan plan = gemm_i8_plan(a.M, a.N, a.K, a.acc != nullptr);
-#ifdef RUDDER_ROLE_PROF
-    const bool dump = false;                        // the dump pointer carries counters in this build
-#else
     const bool dump = a.acc != nullptr;
-#endif
     switch (plan.token_tile) {
         case 32:  return dump ? launch_one<32, true>(a, plan, st) : launch_one<32, false>(a, plan, st);
         case 64:  return dump ? launch_one<64, true>(a, plan, st) : launch_one<64, false>(a, plan, st);
