@@ -167,8 +167,12 @@ rudder_status rudder_block_profile(const rudder_block_args* args, int M, const r
 /* rudder_block for callers whose activations live in HOST memory (pinned for asynchronous copies):
  * args->x[l] and args->y[l] are HOST pointers here (rows contiguous: ldx[l] >= K_l, ldy[l] >= N_l);
  * everything else is as in rudder_block.  Each input is copied to `staging`, the block runs, each
- * output is copied back, all on `stream`, without synchronising.  staging: device memory of at
- * least rudder_block_host_staging_bytes(args, M) bytes, 256-byte aligned. */
+ * output is copied back, without synchronising: work queued on `stream` before the call precedes it,
+ * work queued after the call follows the last copy.  Inside, uploads and downloads run on two
+ * library-owned streams (created on first use, one pair per device) so that they overlap each other
+ * and the kernels; concurrent host threads must therefore not call this on the same device.
+ * staging: device memory of at least rudder_block_host_staging_bytes(args, M) bytes, 256-byte
+ * aligned. */
 size_t rudder_block_host_staging_bytes(const rudder_block_args* args, int M);
 rudder_status rudder_block_host(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
                                 void* staging, size_t staging_bytes, void* workspace, size_t workspace_bytes,

@@ -446,6 +446,35 @@ rudder_status rudder_block_profile(const rudder_block_args* args, int M, const r
     return s;
 }
 
+// Copy streams and events of rudder_block_host, one set per device, created on first use.  Calls on one
+// device share them: concurrent host threads must not call rudder_block_host on the same device.
+struct HostPipe {
+    cudaStream_t in, out;
+    cudaEvent_t start, in_done[4], lin_done[4], out_done;
+    bool ready;
+};
+static HostPipe g_host_pipe[64];
+
+static HostPipe* host_pipe()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPipe* hp = &g_host_pipe[dev];
+    if (!hp->ready) {
+        if (cudaStreamCreateWithFlags(&hp->in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&hp->out, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&hp->start, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&hp->out_done, cudaEventDisableTiming) != cudaSuccess)
+            return nullptr;
+        for (int l = 0; l < 4; ++l)
+            if (cudaEventCreateWithFlags(&hp->in_done[l], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&hp->lin_done[l], cudaEventDisableTiming) != cudaSuccess)
+                return nullptr;
+        hp->ready = true;
+    }
+    return hp;
+}
+
 size_t rudder_block_host_staging_bytes(const rudder_block_args* args, int M)
 {
     if (!args || M < 1) return 0;
@@ -486,20 +515,37 @@ rudder_status rudder_block_host(const rudder_block_args* args, int M, const rudd
         if (s != RUDDER_OK) return s;
     }
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < rudder_block_workspace_bytes(args, M)) return RUDDER_ERR_WORKSPACE;
+    // Uploads, the four linears and downloads run on three streams (PCIe is full duplex): linear l starts
+    // when its input has landed, its output goes back while later inputs are still coming in.  `st` waits
+    // for the last download, so the call keeps the usual stream semantics.
+    HostPipe* hp = host_pipe();
+    if (!hp) return RUDDER_ERR_CUDA;
+    if (cudaEventRecord(hp->start, st) != cudaSuccess || cudaStreamWaitEvent(hp->in, hp->start, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(hp->out, hp->start, 0) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
     for (int l = 0; l < 4; ++l) {
         const int K = args->w[l]->K;
         if (cudaMemcpy2DAsync(const_cast<uint16_t*>(dev.x[l]), static_cast<size_t>(K) * 2, args->x[l], static_cast<size_t>(args->ldx[l]) * 2,
-                              static_cast<size_t>(K) * 2, M, cudaMemcpyHostToDevice, st) != cudaSuccess)
+                              static_cast<size_t>(K) * 2, M, cudaMemcpyHostToDevice, hp->in) != cudaSuccess ||
+            cudaEventRecord(hp->in_done[l], hp->in) != cudaSuccess)
             return RUDDER_ERR_CUDA;
     }
-    rudder_status s = block_impl(&dev, M, seg, step, workspace, workspace_bytes, stream, nullptr);
-    if (s != RUDDER_OK) return s;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
     for (int l = 0; l < 4; ++l) {
         const int N = args->w[l]->N;
-        if (cudaMemcpy2DAsync(args->y[l], static_cast<size_t>(args->ldy[l]) * 2, dev.y[l], static_cast<size_t>(N) * 2,
-                              static_cast<size_t>(N) * 2, M, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        const size_t bytes = workspace_bytes_for(args->w[l], M);
+        if (cudaStreamWaitEvent(st, hp->in_done[l], 0) != cudaSuccess) return RUDDER_ERR_CUDA;
+        rudder_status s = linear_impl(dev.w[l], dev.x[l], dev.ldx[l], M, seg, step, dev.tab[l], dev.bias[l], dev.y[l], dev.ldy[l],
+                                      ws, bytes, st, nullptr, 0, 0, 0, 0, nullptr);
+        if (s != RUDDER_OK) return s;
+        ws += bytes;
+        if (cudaEventRecord(hp->lin_done[l], st) != cudaSuccess || cudaStreamWaitEvent(hp->out, hp->lin_done[l], 0) != cudaSuccess ||
+            cudaMemcpy2DAsync(args->y[l], static_cast<size_t>(args->ldy[l]) * 2, dev.y[l], static_cast<size_t>(N) * 2,
+                              static_cast<size_t>(N) * 2, M, cudaMemcpyDeviceToHost, hp->out) != cudaSuccess)
             return RUDDER_ERR_CUDA;
     }
+    if (cudaEventRecord(hp->out_done, hp->out) != cudaSuccess || cudaStreamWaitEvent(st, hp->out_done, 0) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
     return RUDDER_OK;
 }
 

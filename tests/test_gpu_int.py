@@ -165,6 +165,19 @@ def test_block_matches_four_linears(rd):
         out = oracle.rudder_linear(l.X_bf16, ref_w, l.gamma, None, 1, 0, l.seg_offsets, l.seg_stream, "w4a8", l.bias)
         check_output(bf16_to_np(y), out["y64"])
         assert torch.equal(y, rd.rudder_linear(g.w, g.X, g.seg, 1, g.tab, g.bias))
+    # the same block from pinned host buffers (uploads, kernels and downloads overlap on three streams),
+    # twice in a row over the same staging area
+    xh = [g.X.cpu().pin_memory() for g in gs]
+    yh = [torch.zeros((M, l.N), dtype=torch.bfloat16).pin_memory() for l in lins]
+    hargs = rd.BlockArgs([g.w for g in gs], [g.tab for g in gs], [g.bias for g in gs], xh, yh)
+    staging = torch.empty(rd.rudder_block_host_staging_bytes(hargs, M) + 256, dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        for t in yh:
+            t.zero_()
+        rd.rudder_block_host(hargs, M, gs[0].seg, 1, staging, ws)
+        torch.cuda.current_stream().synchronize()          # the stream waits for the last download
+        for y, t in zip(ys, yh):
+            assert torch.equal(y.cpu(), t)
     _assert_clean(rd)
 
 
