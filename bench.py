@@ -9,7 +9,7 @@ action) tokens, 10 steps of tables).  The W4A8 block (configuration 2), the W4A4
 (configuration 3) and the small-M sweep (configuration 4) are measured in the same run and reported
 under "also" (rank 0, N = 1).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg3_nvfp4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg3_nvfp4|cfg4] [--impl reference]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded row sample.
 """
@@ -226,13 +226,13 @@ def roofline_of(cfg, m, pk):
             "per_kernel_ms": [float(v) for v in m["prof"]]}
 
 
-def small_m_sweep(rd, torch, dev, pk):
+def small_m_sweep(rd, torch, dev, pk, schemes=("w4a8", "w4a4"), sizes=(2048, 4096), rows=(16, 64, 128, 256)):
     """Configuration 4: action + proprio-only passes; one packed weight reused across 20 steps, captured
     in one CUDA graph (weights stay L2-resident: `algorithmic` GB/s counts every byte the call must move)."""
     out = []
-    for scheme in ("w4a8", "w4a4"):
-        for KN in (2048, 4096):
-            for M in (16, 64, 128, 256):
+    for scheme in schemes:
+        for KN in sizes:
+            for M in rows:
                 cfg = wl.config(4, scheme, M=M, KN=KN)
                 l = cfg.draw()[0]
                 W = torch.from_numpy(l.W).to(dev)
@@ -292,6 +292,21 @@ def run_ours(args):
     rd.lib()
     pk = peaks()
 
+    if args.workload == "cfg4":
+        # Configuration 4 alone (the small-M sweep that the default run reports under "also"): the command
+        # the ncu summary of the small-M kernels is taken from.  Rank 0 only; the value is the sweep's
+        # mean throughput.
+        if rank == 0:
+            sweep = small_m_sweep(rd, torch, dev, pk, schemes=("w4a8",))
+            mean_us = float(np.mean([r["us_per_linear"] for r in sweep]))
+            print(json.dumps({"metric": "small-M W4A8 linear (configuration 4), mean over M in {16,64,128,256}, K=N in {2048,4096}",
+                              "value": float(np.mean([r["tops"] for r in sweep])), "unit": "TOPS", "n_gpus": 1,
+                              "steps": 20, "warmup": 5, "ms_per_step": mean_us * 1e-3, "higher_is_better": True,
+                              "scaling": "weak", "vs_baseline": None, "dtype": "int8 x int4 -> int32", "data": "synthetic",
+                              "config": {"workload": "cfg4_small_m_sweep"}, "sweep": sweep}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
     cfg = workload_config(args.workload)
     M, T = cfg.M, cfg.T
     sampler = ClockSampler(local_rank) if rank == 0 else None
