@@ -156,6 +156,9 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_word;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the next prologue kernel may start its own set-up
+    // Launched ahead of the prologue kernel's end: everything above is this CTA's own set-up; the codes,
+    // scales and token scales that the roles below read are the prologue's output.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -345,8 +348,7 @@ static cudaError_t launch_fp4_one(const GemmFp4Args& a, cudaStream_t st)
     p.n_tiles = (a.N + fp4::BN - 1) / fp4::BN;
     const int tiles = p.m_tiles * p.n_tiles;
     const int grid = tiles < a.sm_count ? tiles : a.sm_count;
-    fp4::gemm_nvfp4_kernel<TT><<<grid, fp4::NUM_THREADS, T::DYN_SMEM, st>>>(a.tm_x, a.tm_w, a.tm_y, p);
-    return cudaGetLastError();
+    return launch_early(fp4::gemm_nvfp4_kernel<TT>, grid, fp4::NUM_THREADS, T::DYN_SMEM, st, a.tm_x, a.tm_w, a.tm_y, p);
 }
 
 // 256-token tiles once they fill the device; smaller problems get twice the CTAs from 128-token tiles.

@@ -163,6 +163,9 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_word;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the next prologue kernel may start its own set-up
+    // Launched ahead of the prologue kernel's end: everything above is this CTA's own set-up; the codes,
+    // scales and token scales that the roles below read are the prologue's output.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -370,8 +373,8 @@ cudaError_t launch_gemm_fp4_pair(const GemmFp4Args& a, cudaStream_t st)
     if (clusters < 1) clusters = a.sm_count / 2;
     const int tiles = p.m_tiles * p.n_tiles;
     const int pairs = tiles < clusters ? tiles : clusters;
-    fp4::gemm_nvfp4_pair_kernel<<<2 * pairs, fp4::NUM_THREADS, fp4::PAIR_DYN_SMEM, st>>>(a.tm_x, a.tm_w, a.tm_sfx, a.tm_sfw, a.tm_y, p);
-    return cudaGetLastError();
+    return launch_early(fp4::gemm_nvfp4_pair_kernel, 2 * pairs, fp4::NUM_THREADS, fp4::PAIR_DYN_SMEM, st, a.tm_x, a.tm_w, a.tm_sfx,
+                        a.tm_sfw, a.tm_y, p);
 }
 
 }  // namespace rudder
