@@ -467,7 +467,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": res["seconds"] * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "oracle (fp32 / int32 / fp64 on CPU)", "data": "synthetic",
-            "config": {"workload": cfg.name, "scheme": cfg.scheme, "group": cfg.group, "M": cfg.M,
+            "config": {"workload": cfg.name, "scheme": cfg.scheme, "group": 16 if cfg.scheme == "nvfp4" else cfg.group, "M": cfg.M,
                        "linears": {n: [K, N] for n, K, N in cfg.linears}},
             "cpu_baseline": {"kind": "oracle", "cores": res["cores"], "sample": res["sample"], "value": value, "unit": UNIT},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
