@@ -26,14 +26,15 @@
 // Shared memory rings (stage = 128 input channels):
 //   X  [SX][TT tokens][128 B]     int8, swizzled by TMA       full: TMA bytes     empty: umma commit
 //   W  [SW][128 channels][128 B]  int8 x16, swizzled by hand  full: 4 warps       empty: umma commit
-// The output tile [TT tokens][128 channels] bf16 is staged over the X ring once the last MMA is done.
-// Small M (action / proprio-only passes): the token tile shrinks to 32 / 64 / 128 and the K dimension
-// is split over blockIdx.y so that about one CTA per SM streams its own slice of the weights, several
-// stages of packed weights in flight per thread.  Each split writes its fp32 partial tile; the CTA that
-// arrives last at the tile's counter adds the partials in split order (deterministic) and runs the
-// normal output path.  The kernel may be launched with programmatic dependent launch: everything that
-// does not read the prologue's output (barrier set-up, TMEM allocation, weight prefetch) then overlaps
-// the prologue kernel.
+// 256-token tiles: the output tile [256 tokens][128 channels] bf16 is staged over the X ring once the last
+// MMA is done.
+// Small M (up to 256 tokens: action / proprio-only passes): the token tile shrinks to 32 / 64 and the K
+// dimension is split over blockIdx.y so that about one CTA per SM streams its own slice of the
+// weights, several stages of packed weights in flight per thread.  Each split writes its fp32 partial
+// tile [token][channel]; the CTA that arrives last at the tile's counter adds the partials in split
+// order (deterministic) and stores its bf16 results straight from registers.  The kernel is launched
+// with programmatic dependent launch: everything that does not read the prologue's output (barrier
+// set-up, TMEM allocation) overlaps the prologue kernel.
 // TMEM: NBUF = 512 / TT (at most 8) buffers of TT columns x 128 lanes of INT32, one weight group each.
 // acc_full[b]: umma commit; acc_empty[b]: 8 epilogue warps.
 #include "internal.cuh"
@@ -58,10 +59,6 @@ constexpr int EPI_THREADS = 256;
 #define RUDDER_REGS_LO 72
 #define RUDDER_REGS_HI 184
 #endif
-#ifndef RUDDER_REGS_LO128
-#define RUDDER_REGS_LO128 88
-#define RUDDER_REGS_HI128 168
-#endif
 #ifndef RUDDER_CH
 #define RUDDER_CH 32
 #endif
@@ -84,9 +81,9 @@ constexpr int EPI_THREADS = 256;
 #define RUDDER_SLEEP_EPI 0
 #endif
 
-template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256, 128, 64 or 32
-    static constexpr int SX = (TT == 256) ? 4 : (TT == 128) ? 6 : 8;
-    static constexpr int PD = (TT <= 64) ? 4 : (TT == 128 ? 2 : 1);   // stages of packed weights a thread keeps in flight
+template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256, 64 or 32
+    static constexpr int SX = (TT == 256) ? 4 : 8;
+    static constexpr int PD = (TT <= 64) ? 4 : 1;    // stages of packed weights a thread keeps in flight
     static constexpr int X_BYTES = TT * KSTAGE;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + SX * X_BYTES;
@@ -228,7 +225,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     if (warp < 8) {
     // The epilogue warpgroups hold TT/2 fp32 accumulators per thread: hand them the registers the
     // producer / MMA / unpack warpgroups do not need.
-    if (TT == 256) reg_dec<RUDDER_REGS_LO>(); else if (TT == 128) reg_dec<RUDDER_REGS_LO128>();
+    if (TT == 256) reg_dec<RUDDER_REGS_LO>();
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (activations)
         if (lane == 0) {
@@ -376,7 +373,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     }
     } else {
         // ------------------------------------------------------------------ epilogue
-        if (TT == 256) reg_inc<RUDDER_REGS_HI>(); else if (TT == 128) reg_inc<RUDDER_REGS_HI128>();
+        if (TT == 256) reg_inc<RUDDER_REGS_HI>();
         constexpr int EC = T::EC;
         constexpr int CH = T::CH;                // tokens per TMEM load
         constexpr int NCH = EC / CH;
@@ -650,17 +647,15 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
 GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump)
 {
     GemmI8Plan plan;
-    plan.token_tile = M > 128 ? 256 : (M > 32 ? 64 : 32);
+    plan.token_tile = M > 256 ? 256 : (M > 32 ? 64 : 32);    // up to 256 tokens: small tiles, eight TMEM buffers
     plan.splitk = 1;
     plan.pdl = false;
     if (dump || M > 256) return plan;
     const int n_tiles = (N + BN - 1) / BN;
-    if (M > 128 && n_tiles < 74) plan.token_tile = 128;       // two token tiles double the CTAs
     const int m_tiles = (M + plan.token_tile - 1) / plan.token_tile;
     const int base = m_tiles * n_tiles;
     const size_t m_pad = static_cast<size_t>(m_tiles) * plan.token_tile;
     int sk = 1;
-    if (plan.token_tile > 64) { plan.pdl = true; return plan; }     // K is split for tiles of 32 / 64 tokens only
     while (sk < 16 && base * (sk * 2) <= 160 && (K / KSTAGE) % (sk * 2) == 0 && K / (sk * 2) >= 2 * KSTAGE &&
            static_cast<size_t>(sk * 2) * N * m_pad * sizeof(float) <= (size_t(2) << 20))
         sk *= 2;
@@ -688,8 +683,8 @@ cudaError_t gemm_i8_init()
 #define RUDDER_I8_ATTR(TT, D)                                                                                          \
     e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT>::DYN_SMEM); \
     if (e != cudaSuccess) return e;
-    RUDDER_I8_ATTR(32, false) RUDDER_I8_ATTR(64, false) RUDDER_I8_ATTR(128, false) RUDDER_I8_ATTR(256, false)
-    RUDDER_I8_ATTR(32, true) RUDDER_I8_ATTR(64, true) RUDDER_I8_ATTR(128, true) RUDDER_I8_ATTR(256, true)
+    RUDDER_I8_ATTR(32, false) RUDDER_I8_ATTR(64, false) RUDDER_I8_ATTR(256, false)
+    RUDDER_I8_ATTR(32, true) RUDDER_I8_ATTR(64, true) RUDDER_I8_ATTR(256, true)
 #undef RUDDER_I8_ATTR
     return cudaSuccess;
 }
@@ -701,7 +696,6 @@ cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st)
     switch (plan.token_tile) {
         case 32:  return dump ? launch_one<32, true>(a, plan, st) : launch_one<32, false>(a, plan, st);
         case 64:  return dump ? launch_one<64, true>(a, plan, st) : launch_one<64, false>(a, plan, st);
-        case 128: return dump ? launch_one<128, true>(a, plan, st) : launch_one<128, false>(a, plan, st);
         default:  return dump ? launch_one<256, true>(a, plan, st) : launch_one<256, false>(a, plan, st);
     }
 }
