@@ -508,11 +508,7 @@ static cudaError_t launch_early(void (*kernel)(KArgs...), int grid, int block, s
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-#ifdef RUDDER_DBG_NO_K1PDL
-    cfg.numAttrs = 0;
-#else
     cfg.numAttrs = 1;
-#endif
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 

@@ -54,32 +54,15 @@ constexpr int NUM_THREADS = 512;
 constexpr int UNPACK_THREADS = 128;
 constexpr int EPI_THREADS = 256;
 
-// Back-off (ns) between polls of a barrier, per role.
-#ifndef RUDDER_REGS_LO
-#define RUDDER_REGS_LO 72
-#define RUDDER_REGS_HI 184
-#endif
-#ifndef RUDDER_CH
-#define RUDDER_CH 32
-#endif
-#ifndef RUDDER_EPI_BATCH
-#define RUDDER_EPI_BATCH 1
-#endif
-#ifndef RUDDER_EPI_DB
-#define RUDDER_EPI_DB 1
-#endif
-#ifndef RUDDER_SLEEP_PROD
-#define RUDDER_SLEEP_PROD 64
-#endif
-#ifndef RUDDER_SLEEP_UNPACK
-#define RUDDER_SLEEP_UNPACK 64
-#endif
-#ifndef RUDDER_SLEEP_MMA
-#define RUDDER_SLEEP_MMA 0
-#endif
-#ifndef RUDDER_SLEEP_EPI
-#define RUDDER_SLEEP_EPI 0
-#endif
+// Registers per thread after setmaxnreg (256-token tiles): the drain warps hold 128 accumulators each.
+constexpr int RUDDER_REGS_LO = 72;
+constexpr int RUDDER_REGS_HI = 184;
+// Back-off (ns) between polls of a barrier, per role: the roles that are rarely on the critical path
+// sleep between polls so that they do not take issue slots from the warps that share their scheduler.
+constexpr int RUDDER_SLEEP_PROD = 64;
+constexpr int RUDDER_SLEEP_UNPACK = 64;
+constexpr int RUDDER_SLEEP_MMA = 0;
+constexpr int RUDDER_SLEEP_EPI = 0;
 
 template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256, 64 or 32
     static constexpr int SX = (TT == 256) ? 4 : 8;
@@ -218,9 +201,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     tcgen05_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     volatile int* abortp = &abort_word;
-#ifndef RUDDER_DBG_NO_TRIGGER
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the next prologue kernel may start its own set-up
-#endif
 
     if (warp < 8) {
     // The epilogue warpgroups hold TT/2 fp32 accumulators per thread: hand them the registers the
@@ -450,25 +431,15 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             tcgen05_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * TT + h * EC;
             uint32_t c0[CH], c1[CH];
-#if RUDDER_EPI_DB
             tmem_ld_chunk(taddr, c0);
-#endif
 #pragma unroll
             for (int ch = 0; ch < NCH; ++ch) {
-#if RUDDER_EPI_DB
                 tmem_wait_ld();
                 if (ch + 1 < NCH) {
                     if (ch & 1) tmem_ld_chunk(taddr + (ch + 1) * CH, c0);
                     else        tmem_ld_chunk(taddr + (ch + 1) * CH, c1);
                 }
                 const uint32_t (&cur)[CH] = (ch & 1) ? c1 : c0;
-#else
-                tmem_ld_chunk(taddr + ch * CH, c0);
-                tmem_wait_ld();
-                const uint32_t (&cur)[CH] = c0;
-                (void)c1;
-#endif
-#if RUDDER_EPI_BATCH
                 // Convert the whole chunk first, then accumulate: every FMA then finds its operand ready
                 // instead of waiting out the conversion latency element by element.
                 float f[CH];
@@ -476,11 +447,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 for (int j = 0; j < CH; ++j) asm volatile("cvt.rn.f32.s32 %0, %1;" : "=f"(f[j]) : "r"(cur[j]));
 #pragma unroll
                 for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[ch * CH + j]) : "f"(f[j]), "f"(sc));
-#else
-#pragma unroll
-                for (int j = 0; j < CH; ++j)
-                    acc[ch * CH + j] = fmaf(__int2float_rn(static_cast<int>(cur[j])), sc, acc[ch * CH + j]);
-#endif
                 if (DUMP) {
                     const int cc = n - p.aux.dump.col0;
                     if (p.aux.dump.acc != nullptr && n_ok && cc >= 0 && cc < p.aux.dump.cols) {
