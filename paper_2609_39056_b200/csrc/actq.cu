@@ -474,8 +474,9 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
                 const f32x2 rb2 = pack2(rb, rb);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) { mul2(u[i][k], g2); mul2(u[i][k], inv2); mul2(u[i][k], rb2); }
-                const uint32_t lo = e2m1x8(&u[i][0]);
-                const uint32_t hi = e2m1x8(&u[i][4]);
+                uint32_t lo = e2m1x8(&u[i][0]);
+                uint32_t hi = e2m1x8(&u[i][4]);
+                if (sb == 0u) { lo = 0u; hi = 0u; }    // a block whose scale is zero holds +0 codes, not -0 for negative inputs
                 if (kb < n_blocks) {
                     *reinterpret_cast<uint2*>(static_cast<uint8_t*>(o.codes) + static_cast<size_t>(row) * o.ldc + kb * 8) = make_uint2(lo, hi);
                     o.sf[sf_row + sf_col[i]] = static_cast<uint8_t>(sb);

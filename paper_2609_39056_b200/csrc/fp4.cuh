@@ -53,6 +53,7 @@ __device__ __forceinline__ uint32_t nvfp4_encode_block(const float (&u)[16], uin
     }
     lo = f32x8_to_e2m1(a);
     hi = f32x8_to_e2m1(b);
+    if (sb == 0u) { lo = 0u; hi = 0u; }        // a block whose scale is zero holds +0 codes, not -0 for negative inputs
     return sb;
 }
 

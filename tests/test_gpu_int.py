@@ -46,6 +46,24 @@ def test_pack_without_channel_scales(rd):
     assert np.array_equal(ex["dinv"].cpu().numpy(), np.ones(256, np.float32))
 
 
+def test_pack_degenerate_weights(rd):
+    """Zero row, zero group, a group of tiny negative weights (fp16 scale underflows), one dominant weight,
+    weights exactly on rounding ties of the 4-bit grid."""
+    inp = wl.tiny(seed=131, M=4, K=512, N=64)
+    inp.W[5, :] = 0.0
+    inp.W[3, 64:128] = 0.0
+    inp.W[7, 128:192] = -1e-12
+    inp.W[9, 100] = 3.0
+    inp.W[11, 0:64] = np.tile(np.array([7.0, 3.5, 2.5, 1.5, 0.5, -0.5, -2.5, -6.5], np.float32), 8) * 0.01
+    inp.d[:] = 1.0
+    ref = oracle.pack_int4(inp.W, inp.d, 64)
+    g = GpuLinear(rd, inp, "w4a8", 64)
+    ex = rd.rudder_weight_export(g.w)
+    assert np.array_equal(ex["scales"].cpu().numpy().view(np.uint16), ref["scales"].view(np.uint16))
+    assert np.array_equal(ex["codes"].cpu().numpy(), ref["packed"])
+    _assert_clean(rd)
+
+
 @pytest.mark.parametrize("scheme,qmax", [("w4a8", 127), ("w4a4", 7)])
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("M,K", [(1, 128), (37, 384), (130, 1024), (64, 2048), (19, 4096), (9, 8192), (5, 12288),

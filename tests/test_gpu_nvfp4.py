@@ -42,6 +42,21 @@ def test_pack_export_bit_exact(rd, N, K):
     _assert_clean(rd)
 
 
+def test_pack_degenerate_weights(rd):
+    """Zero row, zero block, a block of tiny negative weights whose scale rounds to zero, one dominant weight."""
+    inp = wl.tiny(seed=431, M=4, K=512, N=64)
+    inp.W[5, :] = 0.0
+    inp.W[3, 16:32] = 0.0
+    inp.W[7, 32:48] = -1e-9
+    inp.W[9, 100] = 3.0
+    ref = oracle.pack_nvfp4(inp.W, inp.d)
+    g = GpuLinear(rd, inp, "nvfp4", 16)
+    ex = rd.rudder_weight_export(g.w)
+    assert np.array_equal(ex["scales"].cpu().numpy(), ref["sb"])
+    assert np.array_equal(ex["codes"].cpu().numpy(), ref["packed"])
+    _assert_clean(rd)
+
+
 @pytest.mark.parametrize("mode", [0, 1])
 @pytest.mark.parametrize("M,K", [(1, 256), (37, 512), (130, 1024), (64, 2048), (19, 4096), (9, 8192), (5, 12288),
                                  (300, 3072), (3, 16640)])   # many rows per CTA; rows too long to stage (warp-per-row kernel)
@@ -57,6 +72,38 @@ def test_activation_codes_bit_exact(rd, mode, M, K):
         assert np.array_equal(sb.cpu().numpy(), rsb), "block scales differ"
         assert np.array_equal(codes.cpu().numpy(), _pack_codes(re)), "E2M1 codes differ"
         assert np.array_equal(r.cpu().numpy().view(np.uint32), rr.view(np.uint32))
+    _assert_clean(rd)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_activation_degenerate_rows(rd, mode):
+    """Zero row, one non-zero element, an all-zero 16-channel block, one huge outlier among tiny values,
+    values at the bottom of the bf16 range, equal magnitudes (every rounding tie the formats have)."""
+    K = 512
+    inp = wl.tiny(seed=577, M=8, K=K, N=64, T=2)
+    X = wl.bf16_bits_to_f32(inp.X_bf16).copy()
+    X[0, :] = 0.0
+    X[1, :] = 0.0; X[1, 77] = -3.5
+    X[2, 32:48] = 0.0
+    X[3, :] *= 1e-3; X[3, 5] = 1.0e4
+    X[4, :] *= 1e-30
+    X[5, :] = np.where(np.arange(K) % 2 == 0, 1.0, -1.0)
+    X[6, :] = np.tile(np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0], np.float32), K // 8)   # E2M1 midpoints before scaling
+    inp.X_bf16[:] = wl.f32_to_bf16_bits(X)
+    ref_w = oracle.pack_nvfp4(inp.W, inp.d)
+    clip = static_clip(inp, ref_w["dinv"]) if mode == 1 else None
+    g = GpuLinear(rd, inp, "nvfp4", 16, mode, clip)
+    for step in (0, 1):
+        codes, sb, r = rd.rudder_quantize_activations(g.w, g.X, g.seg, step, g.tab)
+        re, rsb, rr = oracle.quantize_nvfp4(inp.X_bf16, ref_w["dinv"], inp.gamma, clip, step, mode, inp.seg_offsets,
+                                            inp.seg_stream)
+        assert np.array_equal(sb.cpu().numpy(), rsb), "block scales differ"
+        assert np.array_equal(codes.cpu().numpy(), _pack_codes(re)), "E2M1 codes differ"
+        assert np.array_equal(r.cpu().numpy().view(np.uint32), rr.view(np.uint32))
+    # and through the GEMM: the zero row gives the bias, nothing is NaN
+    Y = rd.rudder_linear(g.w, g.X, g.seg, 0, g.tab, g.bias)
+    out = oracle.rudder_linear(inp.X_bf16, ref_w, inp.gamma, clip, 0, mode, inp.seg_offsets, inp.seg_stream, "nvfp4", inp.bias)
+    check_output(bf16_to_np(Y), out["y64"], rel=REL_TOL_FP4, abs_=ABS_TOL)
     _assert_clean(rd)
 
 
