@@ -9,7 +9,7 @@ action) tokens, 10 steps of tables).  The W4A8 block (configuration 2), the W4A4
 (configuration 3) and the small-M sweep (configuration 4) are measured in the same run and reported
 under "also" (rank 0, N = 1).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3|cfg3_nvfp4|cfg4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg2_g128|cfg2_perchannel|cfg3|cfg3_nvfp4|cfg4] [--impl reference]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded row sample.
 """
@@ -52,6 +52,11 @@ def workload_config(name: str):
         return wl.config(3, "w4a4")
     if name == "cfg3_nvfp4":
         return wl.config(3, "nvfp4")
+    if name in ("cfg2_g128", "cfg2_perchannel"):      # configuration 2 at the other weight-scale granularities
+        import dataclasses
+        c = wl.config(2)
+        g = 128 if name == "cfg2_g128" else 0         # 0: one scale per output channel (Eq. 10 as printed)
+        return dataclasses.replace(c, name=c.name + ("_g128" if g else "_per_channel"), group=g)
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -63,7 +68,7 @@ def algorithmic_bytes_linear(M, K, N, G, scheme):
         w = N * K // 2 + N * K // 16 + 4
     else:
         act = M * K + 4 * M           # one code per byte in the workspace (both integer schemes)
-        w = N * K // 2 + 2 * N * K // G
+        w = N * K // 2 + 2 * N * K // (G or K)       # G = 0: one scale per output channel
     return 2 * M * K + 2 * act + w + 2 * M * N + 4 * N
 
 
@@ -130,7 +135,7 @@ def build_block(rd, cfg, torch, dev):
     for l in lins:
         W = torch.from_numpy(l.W).to(dev)
         d = torch.from_numpy(l.d).to(dev)
-        ws.append(rd.rudder_pack_weights(W, d, scheme, cfg.group))
+        ws.append(rd.rudder_pack_weights(W, d, scheme, cfg.group or l.K))     # group 0: one scale per output channel (G = K)
         del W, d
         gamma = torch.from_numpy(l.gamma).to(dev)
         tabs.append(rd.ScaleTable(gamma, None, rd.RANGE_PER_TOKEN))
@@ -378,7 +383,7 @@ def run_ours(args):
         del m, ws, tabs, biases, xs, ys, workspace, lins
         torch.cuda.empty_cache()
         also = {}
-        for name in ("cfg2", "cfg3", "cfg3_nvfp4"):
+        for name in ("cfg2", "cfg2_g128", "cfg2_perchannel", "cfg3", "cfg3_nvfp4"):
             if name == args.workload:
                 continue
             c2 = workload_config(name)
@@ -426,7 +431,7 @@ def cpu_baseline(cfg, lins, target_s=15.0, impl_reference=False):
     cores = oracle.num_threads()
     packs = []
     for l in lins:
-        packs.append(oracle.pack_nvfp4(l.W, l.d) if cfg.scheme == "nvfp4" else oracle.pack_int4(l.W, l.d, cfg.group))
+        packs.append(oracle.pack_nvfp4(l.W, l.d) if cfg.scheme == "nvfp4" else oracle.pack_int4(l.W, l.d, cfg.group or l.K))
     M = cfg.M
 
     def run(rows):
