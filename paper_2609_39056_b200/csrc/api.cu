@@ -216,7 +216,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
                       static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128), box_tok,
                       CU_TENSOR_MAP_SWIZZLE_NONE))
         return RUDDER_ERR_CUDA;
-    g.w_codes = w->codes; g.w_scales_t = w->scales_t;
+    g.w_codes = w->codes; g.w_scales_t = w->scales_t; g.tm_w = w->tm_codes;
     g.y = Y; g.ldy = ldy;
     g.M = M; g.N = w->N; g.K = w->K; g.G = w->G;
     g.row_scale = r; g.bias = bias;
@@ -305,6 +305,14 @@ rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, 
              cudaStreamSynchronize(st) == cudaSuccess;
     }
     if (tmp) cudaFree(tmp);
+    if (ok) {
+        // tensor map over the packed codes, kept in device memory so that the GEMM takes it by pointer
+        CUtensorMap tm;
+        ok = make_tmap_2d(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w->codes, static_cast<uint64_t>(K / 2), static_cast<uint64_t>(N),
+                          static_cast<uint64_t>(K / 2), 64, static_cast<uint32_t>(N < 128 ? N : 128), CU_TENSOR_MAP_SWIZZLE_NONE) &&
+             cudaMalloc(&w->tm_codes, sizeof(CUtensorMap)) == cudaSuccess &&
+             cudaMemcpy(w->tm_codes, &tm, sizeof(CUtensorMap), cudaMemcpyHostToDevice) == cudaSuccess;
+    }
     if (!ok) {
         rudder_weight_free(w);
         return RUDDER_ERR_CUDA;
@@ -322,6 +330,7 @@ rudder_status rudder_weight_free(rudder_weight* w)
     cudaFree(w->sf_tiled);
     cudaFree(w->dinv);
     cudaFree(w->tensor_scale);
+    cudaFree(w->tm_codes);
     free(w);
     return RUDDER_OK;
 }

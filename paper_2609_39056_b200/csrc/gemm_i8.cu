@@ -12,9 +12,11 @@
 // Warp roles (warpgroup-aligned so that registers can be moved between them):
 //   warp 0        TMA producer: activation codes (int8 [TT tokens][128 B], 128-byte swizzle)
 //   warp 1        allocates TMEM; one lane issues tcgen05.mma kind::i8 (M = 128, N = TT, K = 32)
-//   warps 4-7     stream the packed INT4 weights from global memory (L2) into registers one stage
-//                 ahead, expand them to int8 and store them in the swizzled K-major layout the tensor
-//                 core reads.  The nibble goes to the TOP half of the byte (value 16 q): two logic ops
+//   warp 3        (256-token tiles) TMA producer of the packed INT4 weights: a ring of raw stages
+//                 [128 channels][64 B], several stages ahead of the unpack warps
+//   warps 4-7     take the packed INT4 weights (256-token tiles: from the raw ring; small tiles: from
+//                 global memory / L2 into registers, several stages ahead), expand them to int8 and store
+//                 them in the swizzled K-major layout the tensor core reads.  The nibble goes to the TOP half of the byte (value 16 q): two logic ops
 //                 per 8 weights, no sign extension; the factor 16 is folded into the fp32 scales.
 //   warps 8-15    epilogue: per weight group, drain the INT32 partial sums from TMEM and accumulate
 //                 fp32(C) * Delta_W[j,g] in registers; finally * r_i + b_j -> bf16, transposed through
@@ -26,6 +28,7 @@
 // Shared memory rings (stage = 128 input channels):
 //   X  [SX][TT tokens][128 B]     int8, swizzled by TMA       full: TMA bytes     empty: umma commit
 //   W  [SW][128 channels][128 B]  int8 x16, swizzled by hand  full: 4 warps       empty: umma commit
+//   RAW[SR][128 channels][64 B]   packed INT4, as in memory   full: TMA bytes     empty: 4 warps  (256-token tiles)
 // 256-token tiles: the output tile [256 tokens][128 channels] bf16 is staged over the X ring once the last
 // MMA is done.
 // Small M (up to 256 tokens: action / proprio-only passes): the token tile shrinks to 32 / 64 and the K
@@ -50,6 +53,8 @@ constexpr int BN = 128;          // output channels per tile (MMA M)
 constexpr int KSTAGE = 128;      // input channels (= bytes of int8 per row) per pipeline stage
 constexpr int SW = 4;            // unpacked-weight stages
 constexpr int W_BYTES = BN * KSTAGE;
+constexpr int SR = 4;            // packed-weight stages (256-token tiles)
+constexpr int RAW_BYTES = BN * KSTAGE / 2;
 constexpr int NUM_THREADS = 512;
 constexpr int UNPACK_THREADS = 128;
 constexpr int EPI_THREADS = 256;
@@ -70,7 +75,9 @@ template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256, 6
     static constexpr int X_BYTES = TT * KSTAGE;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + SX * X_BYTES;
-    static constexpr int BYTES = OFF_W + SW * W_BYTES;
+    static constexpr bool RAW = (TT == 256);         // packed weights staged by TMA (one more ring) instead of registers
+    static constexpr int OFF_RAW = OFF_W + SW * W_BYTES;
+    static constexpr int BYTES = OFF_RAW + (RAW ? SR * RAW_BYTES : 0);
     static constexpr int DYN_SMEM = BYTES + 1024;    // slack to align the base to 1024 bytes
     static constexpr int NBUF = (512 / TT > 8) ? 8 : 512 / TT;   // TMEM accumulator buffers (one weight group each)
     static constexpr int TMEM_COLS = NBUF * TT;
@@ -94,17 +101,21 @@ struct Params {
     int m_tiles, n_tiles;        // token tiles, channel tiles (grid.x = m_tiles * n_tiles)
     int splitk;                  // K splits (grid.y)
     int stages_per_split;        // 128-channel stages per split
-    float* partials;             // [splitk][m_tiles * TT][N] fp32 partial sums (splitk > 1)
+    union {                      // (shared storage for the same reason as above: a launch uses one of them)
+        float* partials;         // tiles of 32 / 64 tokens: [splitk][m_tiles * TT][N] fp32 partial sums (splitk > 1)
+        const CUtensorMap* tm_w; // 256-token tiles: tensor map (device memory) over the packed weights, box {64 B, 128 channels}
+    };
     int* counters;               // [m_tiles * n_tiles] arrivals per tile, zeroed by the prologue kernel
     int pdl;                     // launched with programmatic dependent launch
     uint32_t x_tx;               // bytes one activation TMA box delivers
     int out_pitch;               // channels per row of the staged output tile (= TMA store box width)
+    uint32_t w_tx;               // bytes one packed-weight TMA box delivers (256-token tiles)
 };
-
+static_assert(sizeof(Params) <= 120, "kernel parameters beyond 376 bytes slow the 256-token kernel");
 
 enum Where {   // codes recorded when a bounded wait gives up
-    W_X_EMPTY = 101,
-    W_W_EMPTY = 201,
+    W_X_EMPTY = 101, W_RAW_EMPTY = 102,
+    W_W_EMPTY = 201, W_RAW_FULL = 202,
     W_X_FULL = 301, W_W_FULL = 302, W_ACC_EMPTY = 303,
     W_ACC_FULL = 401, W_RS_FULL = 402
 };
@@ -117,6 +128,11 @@ __device__ __forceinline__ void sts128(uint32_t addr, const uint4& v) {
 // too and keep their place relative to the stores.
 __device__ __forceinline__ void sts16(uint32_t addr, uint16_t v) {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
 }
 __device__ __forceinline__ uint4 ldg_nc_16(const void* p) {
     uint4 v;
@@ -154,7 +170,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 {
     using T = Tile<TT>;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * SW + 2 * T::NBUF + 1];
+    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * SW + 2 * T::NBUF + 1 + 2 * SR];
     __shared__ __align__(16) float rs_smem[TT];      // row scales r_i of the tile's tokens (0 past M)
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_word;
@@ -183,6 +199,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     auto acc_full = [&](int i) { return bar0 + 8u * (2 * T::SX + 2 * SW + i); };
     auto acc_empty = [&](int i) { return bar0 + 8u * (2 * T::SX + 2 * SW + T::NBUF + i); };
     const uint32_t rs_full = bar0 + 8u * (2 * T::SX + 2 * SW + 2 * T::NBUF);
+    auto raw_full = [&](int i) { return rs_full + 8u * (1 + i); };
+    auto raw_empty = [&](int i) { return rs_full + 8u * (1 + SR + i); };
 
     if (threadIdx.x == 0) {
         abort_word = 0;
@@ -190,6 +208,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         for (int i = 0; i < SW; ++i) { mbar_init(w_full(i), UNPACK_THREADS / 32); mbar_init(w_empty(i), 1); }
         for (int i = 0; i < T::NBUF; ++i) { mbar_init(acc_full(i), 1); mbar_init(acc_empty(i), EPI_THREADS / 32); }
         mbar_init(rs_full, 1);
+        if (T::RAW)
+            for (int i = 0; i < SR; ++i) { mbar_init(raw_full(i), 1); mbar_init(raw_empty(i), UNPACK_THREADS / 32); }
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -287,6 +307,29 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         for (int i = lane; i < TT; i += 32) rs_smem[i] = (m0 + i < p.M) ? ld_f32_volatile(p.row_scale + m0 + i) : 0.0f;
         __syncwarp();
         if (lane == 0) mbar_arrive(rs_full);
+    } else if (warp == 3) {
+        // ------------------------------------------------------------------ TMA producer (packed weights)
+        // The weights do not depend on the prologue kernel: this stream starts at once.  Channels past N
+        // are zero-filled by the copy.
+        if (T::RAW && lane == 0) {
+            tma_prefetch_desc(p.tm_w);
+            int issued = 0;
+            bool ok = true;
+            int slot = 0;
+            uint32_t ph = 0;
+            for (int s = 0; s < n_stages; ++s) {
+                ok = mbar_wait<RUDDER_SLEEP_PROD>(raw_empty(slot), ph ^ 1u, abortp, W_RAW_EMPTY);
+                if (!ok) break;
+                mbar_expect_tx(raw_full(slot), p.w_tx);
+                tma_load_2d(smem_base + T::OFF_RAW + slot * RAW_BYTES, p.tm_w, (s0 + s) * (KSTAGE / 2), n0, raw_full(slot));
+                ++issued;
+                if (++slot == SR) { slot = 0; ph ^= 1u; }
+            }
+            if (!ok) {
+                for (int i = max(0, issued - SR); i < issued; ++i)
+                    for (uint32_t it = 0; it < (1u << 16) && !mbar_try_wait(raw_full(i % SR), (i / SR) & 1); ++it) {}
+            }
+        }
     } else if (warp >= 4) {
         // ------------------------------------------------------------------ INT4 -> int8 unpack
         // 128 channels x 64 packed bytes per stage = 512 16-byte pieces, 4 per thread: piece idx covers
@@ -304,6 +347,44 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         }
         // PD stages of packed weights are in flight per thread (registers), so that the L2 / DRAM latency
         // of the weight stream is covered even when a stage is consumed quickly.
+        if (T::RAW) {
+            bool ok = true;
+            int sw = 0, sr = 0;
+            uint32_t phw = 0, phr = 0;
+            for (int s = 0; s < n_stages && ok; ++s) {
+                ok = mbar_wait<RUDDER_SLEEP_UNPACK>(raw_full(sr), phr, abortp, W_RAW_FULL);
+                if (!ok) break;
+                uint4 cur[4];
+                const uint32_t rsrc = smem_base + T::OFF_RAW + sr * RAW_BYTES;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    cur[i] = lds128(rsrc + (i * UNPACK_THREADS + tid) * 16);
+                    if (!valid[i]) cur[i] = make_uint4(0, 0, 0, 0);
+                }
+                ok = mbar_wait<RUDDER_SLEEP_UNPACK>(w_empty(sw), phw ^ 1u, abortp, W_W_EMPTY);
+                if (!ok) break;
+                const uint32_t dst = smem_base + T::OFF_W + sw * W_BYTES;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int idx = i * UNPACK_THREADS + tid;
+                    const int row = idx >> 2, ch = idx & 3;
+                    const uint4 pk = cur[i];
+                    uint4 lo, hi;
+                    lo.x = (pk.x << 4) & 0xF0F0F0F0u; hi.x = pk.x & 0xF0F0F0F0u;
+                    lo.y = (pk.y << 4) & 0xF0F0F0F0u; hi.y = pk.y & 0xF0F0F0F0u;
+                    lo.z = (pk.z << 4) & 0xF0F0F0F0u; hi.z = pk.z & 0xF0F0F0F0u;
+                    lo.w = (pk.w << 4) & 0xF0F0F0F0u; hi.w = pk.w & 0xF0F0F0F0u;
+                    const uint32_t drow = dst + (row >> 3) * 1024 + (row & 7) * 128;
+                    sts128(drow + (((2 * ch) ^ (row & 7)) << 4), lo);
+                    sts128(drow + (((2 * ch + 1) ^ (row & 7)) << 4), hi);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) { mbar_arrive(w_full(sw)); mbar_arrive(raw_empty(sr)); }
+                if (++sw == SW) { sw = 0; phw ^= 1u; }
+                if (++sr == SR) { sr = 0; phr ^= 1u; }
+            }
+        } else {
         constexpr int PD = T::PD;
         uint4 pre[PD][4];
         auto load_stage = [&](int s, uint4 (&dst)[4]) {
@@ -350,6 +431,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     }
                 }
             }
+        }
         }
     }
     } else {
@@ -585,11 +667,12 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
     else      { p.aux.out.y = a.y; p.aux.out.ldy = a.ldy; }
     p.x_tx = static_cast<uint32_t>(min(TT, a.M)) * KSTAGE;
     p.out_pitch = min(BN, a.N);
+    p.w_tx = static_cast<uint32_t>(min(BN, a.N)) * (KSTAGE / 2);
     p.m_tiles = (a.M + TT - 1) / TT;
     p.n_tiles = (a.N + BN - 1) / BN;
     p.splitk = plan.splitk;
     p.stages_per_split = a.K / KSTAGE / plan.splitk;
-    p.partials = a.partials;
+    if (T::RAW) p.tm_w = a.tm_w; else p.partials = a.partials;
     p.counters = a.counters;
     p.pdl = plan.pdl ? 1 : 0;
 

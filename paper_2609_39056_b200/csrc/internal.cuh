@@ -42,6 +42,8 @@ struct rudder_weight {
     uint8_t* sf_tiled;
     float* dinv;
     float* tensor_scale;      // device [1]
+    CUtensorMap* tm_codes;    // integer schemes: tensor map (in device memory) over the packed codes [N, K/2],
+                              // box {64 bytes, 128 channels}: one pipeline stage of one channel tile
     size_t bytes;
 };
 
@@ -100,6 +102,7 @@ struct GemmI8Args {
     CUtensorMap tm_y;           // output bf16 [M, N] (row pitch ldy), box {min(128, N) channels, token tile}
     uint16_t* y;                // the same output as a plain pointer (small tiles are stored without TMA)
     int64_t ldy;
+    const CUtensorMap* tm_w;    // device-resident tensor map over the packed weights (256-token tiles stage them by TMA)
     const uint8_t* w_codes;     // packed INT4 weights
     const float* w_scales_t;    // [K/G][N]
     int M, N, K, G;
