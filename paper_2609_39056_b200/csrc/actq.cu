@@ -43,6 +43,19 @@ __device__ __forceinline__ void scale8(const uint4& x, const float4& d0, const f
     }
 }
 
+// Two integer-valued floats in [-7, 7] -> two E4M3 bytes (exact), lo in the low byte.
+__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+    uint16_t h;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(h) : "f"(hi), "f"(lo));
+    return h;
+}
+__device__ __forceinline__ uint2 round8_e4m3(const float (&v)[8], float inv, int qmax) {
+    const float qf = static_cast<float>(qmax);
+    float q[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = fminf(fmaxf(rintf(__fmul_rn(v[i], inv)), -qf), qf);
+    return make_uint2(e4m3x2(q[0], q[1]) | (e4m3x2(q[2], q[3]) << 16), e4m3x2(q[4], q[5]) | (e4m3x2(q[6], q[7]) << 16));
+}
 __device__ __forceinline__ uint2 round8(const float (&v)[8], float inv, int qmax) {
     uint32_t out[2] = {0u, 0u};
 #pragma unroll
@@ -56,7 +69,7 @@ __device__ __forceinline__ uint2 round8(const float (&v)[8], float inv, int qmax
 
 // NIT = number of 256-channel steps whose raw data is kept in registers (0: re-read the row).
 template <int NIT>
-__global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int8_t* __restrict__ codes, int64_t ldc,
+__global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int e4m3, int8_t* __restrict__ codes, int64_t ldc,
                                                         float* __restrict__ r)
 {
     asm volatile("griddepcontrol.wait;" ::: "memory");     // may have been launched ahead of its stream predecessors
@@ -117,7 +130,7 @@ __global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int
             if (c < n_chunks) {
                 float v[8];
                 scale8(xr[it], __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
-                crow[c] = round8(v, inv, qmax);
+                crow[c] = e4m3 ? round8_e4m3(v, inv, qmax) : round8(v, inv, qmax);
             }
         }
     } else {
@@ -126,7 +139,7 @@ __global__ void __launch_bounds__(256) actq_int_kernel(ActqArgs a, int qmax, int
             if (c < n_chunks) {
                 float v[8];
                 scale8(ld_nc_16(xrow + c), __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
-                crow[c] = round8(v, inv, qmax);
+                crow[c] = e4m3 ? round8_e4m3(v, inv, qmax) : round8(v, inv, qmax);
             }
         }
     }
@@ -256,6 +269,7 @@ struct RowOut {
     float* r;
     int M_pad;
     int qmax;
+    int e4m3;                  // integer codes written as E4M3 bytes
 };
 
 typedef unsigned long long f32x2;                  // two fp32 lanes in one 64-bit register pair
@@ -346,6 +360,20 @@ __device__ __forceinline__ uint2 s8x8(const f32x2* v, float qmaxf) {
     asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(t1) : "r"(q[7]), "r"(q[6]));
     asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q[5]), "r"(q[4]), "r"(t1));
     return make_uint2(lo, hi);
+}
+
+// Four lane pairs -> eight E4M3 bytes holding the rounded integers (|.| <= qmaxf <= 7).
+__device__ __forceinline__ uint2 e4m3x8(const f32x2* v, float qmaxf) {
+    uint32_t h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float lo, hi;
+        unpack2(v[i], lo, hi);
+        lo = fminf(fmaxf(rintf(lo), -qmaxf), qmaxf);
+        hi = fminf(fmaxf(rintf(hi), -qmaxf), qmaxf);
+        h[i] = e4m3x2(lo, hi);
+    }
+    return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
 }
 
 template <bool FP4, int NCH>
@@ -485,8 +513,14 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
 #pragma unroll
                 for (int k = 0; k < 8; ++k) { mul2(u[i][k], g2); mul2(u[i][k], inv2); }
                 const float qmaxf = range_max;
-                const uint2 q0 = per_token ? s8x8<false>(&u[i][0], qmaxf) : s8x8<true>(&u[i][0], qmaxf);
-                const uint2 q1 = per_token ? s8x8<false>(&u[i][4], qmaxf) : s8x8<true>(&u[i][4], qmaxf);
+                uint2 q0, q1;
+                if (o.e4m3) {
+                    q0 = e4m3x8(&u[i][0], qmaxf);
+                    q1 = e4m3x8(&u[i][4], qmaxf);
+                } else {
+                    q0 = per_token ? s8x8<false>(&u[i][0], qmaxf) : s8x8<true>(&u[i][0], qmaxf);
+                    q1 = per_token ? s8x8<false>(&u[i][4], qmaxf) : s8x8<true>(&u[i][4], qmaxf);
+                }
                 if (kb < n_blocks)
                     *reinterpret_cast<uint4*>(static_cast<uint8_t*>(o.codes) + static_cast<size_t>(row) * o.ldc + kb * 16) = make_uint4(q0.x, q0.y, q1.x, q1.y);
             }
@@ -563,7 +597,7 @@ cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bo
 {
     const int M_pad = sf_tiled ? ((a.M + 127) / 128) * 128 : a.M;
     RowOut o;
-    o.codes = codes; o.ldc = a.K / 2; o.sf = sf; o.sf_tiled = sf_tiled ? 1 : 0; o.r = r; o.M_pad = M_pad; o.qmax = 0;
+    o.codes = codes; o.ldc = a.K / 2; o.sf = sf; o.sf_tiled = sf_tiled ? 1 : 0; o.r = r; o.M_pad = M_pad; o.qmax = 0; o.e4m3 = 0;
     cudaError_t err = cudaSuccess;
     if (!launch_row<true>(a, o, M_pad, st, &err)) {
         const int blocks = (M_pad * 32 + 255) / 256;      // unaligned or very long rows: one warp per row, row read twice
@@ -572,15 +606,15 @@ cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bo
     return err != cudaSuccess ? err : cudaGetLastError();
 }
 
-cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st)
+cudaError_t launch_actq_int(const ActqArgs& a, int qmax, bool e4m3, int8_t* codes, int64_t ldc, float* r, cudaStream_t st)
 {
     RowOut o;
-    o.codes = codes; o.ldc = ldc; o.sf = nullptr; o.sf_tiled = 0; o.r = r; o.M_pad = a.M; o.qmax = qmax;
+    o.codes = codes; o.ldc = ldc; o.sf = nullptr; o.sf_tiled = 0; o.r = r; o.M_pad = a.M; o.qmax = qmax; o.e4m3 = e4m3 ? 1 : 0;
     cudaError_t err = cudaSuccess;
     if (!launch_row<false>(a, o, a.M, st, &err)) {
         const int blocks = (a.M * 32 + 255) / 256;         // unaligned or very long rows: one warp per row, row read twice
         if (a.zero_ints != nullptr && cudaMemsetAsync(a.zero_ints, 0, sizeof(int) * a.n_zero, st) != cudaSuccess) return cudaErrorUnknown;
-        err = launch_early(actq_int_kernel<0>, blocks, 256, 0, st, a, qmax, codes, ldc, r);
+        err = launch_early(actq_int_kernel<0>, blocks, 256, 0, st, a, qmax, e4m3 ? 1 : 0, codes, ldc, r);
     }
     return err != cudaSuccess ? err : cudaGetLastError();
 }

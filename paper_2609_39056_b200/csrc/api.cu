@@ -204,7 +204,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
         a.zero_ints = g.counters;
         a.n_zero = ((M + plan.token_tile - 1) / plan.token_tile) * ((w->N + 127) / 128);
     }
-    if (launch_actq_int(a, qmax_of(w->scheme), codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if (launch_actq_int(a, qmax_of(w->scheme), w->f8 != 0, codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
 
     const int tt = plan.token_tile;
@@ -216,7 +216,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
                       static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128), box_tok,
                       CU_TENSOR_MAP_SWIZZLE_NONE))
         return RUDDER_ERR_CUDA;
-    g.w_codes = w->codes; g.w_scales_t = w->scales_t; g.tm_w = w->tm_codes;
+    g.w_codes = w->codes; g.w_scales_t = w->scales_t; g.tm_w = w->tm_codes; g.f8 = w->f8 != 0;
     g.y = Y; g.ldy = ldy;
     g.M = M; g.N = w->N; g.K = w->K; g.G = w->G;
     g.row_scale = r; g.bias = bias;
@@ -290,6 +290,11 @@ rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, 
         *out = w;
         return RUDDER_OK;
     }
+    // W4A4 with group scales: |C^(g)| <= 128 * 49, so E4M3 operands and FP32 accumulators hold the
+    // integers exactly and the per-group drain needs no integer-to-float conversion.
+#ifndef RUDDER_NO_F8
+    w->f8 = (scheme == RUDDER_W4A4_INT && group <= 128) ? 1 : 0;
+#endif
     int8_t* tmp = nullptr;
     bool ok = cudaMalloc(&w->codes, code_bytes) == cudaSuccess &&
               cudaMalloc(&w->scales_t, n_groups * N * sizeof(float)) == cudaSuccess &&
@@ -301,7 +306,7 @@ rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, 
     if (ok) {
         const float one = 1.0f;
         ok = cudaMemcpyAsync(w->tensor_scale, &one, sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess &&
-             launch_pack_int4(W, d, N, K, group, w->codes, w->scales_t, static_cast<uint16_t*>(w->scales_c), w->dinv, tmp, st) == cudaSuccess &&
+             launch_pack_int4(W, d, N, K, group, w->codes, w->scales_t, static_cast<uint16_t*>(w->scales_c), w->dinv, tmp, w->f8 != 0, st) == cudaSuccess &&
              cudaStreamSynchronize(st) == cudaSuccess;
     }
     if (tmp) cudaFree(tmp);
@@ -358,7 +363,7 @@ rudder_status rudder_weight_export(const rudder_weight* w, uint8_t* codes, void*
         if (scales && cudaMemcpyAsync(scales, w->scales_c, n_groups * w->N, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
             return RUDDER_ERR_CUDA;
     } else {
-        if (codes && launch_export_int4(w->codes, w->N, w->K, codes, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (codes && launch_export_int4(w->codes, w->N, w->K, codes, w->f8 != 0, st) != cudaSuccess) return RUDDER_ERR_CUDA;
         if (scales && cudaMemcpyAsync(scales, w->scales_c, n_groups * w->N * sizeof(uint16_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
             return RUDDER_ERR_CUDA;
     }
@@ -581,7 +586,7 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
             return RUDDER_ERR_CUDA;
         return RUDDER_OK;
     }
-    if (launch_actq_int(a, qmax_of(w->scheme), static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    if (launch_actq_int(a, qmax_of(w->scheme), false, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     return RUDDER_OK;
 }

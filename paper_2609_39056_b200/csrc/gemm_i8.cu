@@ -164,7 +164,33 @@ __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wa
 __device__ __forceinline__ void tmem_ld_chunk(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld_32x32b_x32(taddr, r); }
 __device__ __forceinline__ void tmem_ld_chunk(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld_32x32b_x16(taddr, r); }
 
-template <int TT, bool DUMP>
+// Eight packed 4-bit weights -> two words of four operand bytes each.
+// Integer path: two's complement nibbles moved to the top half of the byte (the value 16 q).
+// E4M3 path: sign-magnitude words (see the offline pack); the magnitudes index a table of the E4M3
+// encodings of 0..7 held in two registers (byte permute), the signs are moved to bit 7.
+template <bool F8>
+__device__ __forceinline__ void unpack8(uint32_t pk, uint32_t& lo, uint32_t& hi) {
+    if (F8) {
+        const uint32_t t_lo = 0x44403800u, t_hi = 0x4E4C4A48u;      // E4M3 of 0, 1, 2, 3 and of 4, 5, 6, 7
+        uint32_t ma, mb;
+        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(ma) : "r"(t_lo), "r"(t_hi), "r"(pk & 0x7777u));
+        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(mb) : "r"(t_lo), "r"(t_hi), "r"((pk >> 16) & 0x7777u));
+        lo = ma | ((pk << 4) & 0x80808080u);
+        hi = mb | (pk & 0x80808080u);
+    } else {
+        lo = (pk << 4) & 0xF0F0F0F0u;
+        hi = pk & 0xF0F0F0F0u;
+    }
+}
+template <bool F8>
+__device__ __forceinline__ void unpack32(const uint4& pk, uint4& lo, uint4& hi) {
+    unpack8<F8>(pk.x, lo.x, hi.x);
+    unpack8<F8>(pk.y, lo.y, hi.y);
+    unpack8<F8>(pk.z, lo.z, hi.z);
+    unpack8<F8>(pk.w, lo.w, hi.w);
+}
+
+template <int TT, bool DUMP, bool F8>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y, const Params p)
 {
@@ -257,7 +283,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // registers); one elected lane issues the MMAs and the commits.
         {
             const bool leader = elect_one();
-            const uint32_t idesc = umma_idesc_i8(BN, TT);
+            const uint32_t idesc = F8 ? umma_idesc_e4m3(BN, TT) : umma_idesc_i8(BN, TT);
             bool ok = true;
             // No divisions in this loop: every instruction on this path is latency the tensor core may
             // end up waiting for.
@@ -283,7 +309,10 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                         if (!ok) break;
                         tcgen05_fence_after_sync();
                     }
-                    if (leader) umma_i8(tmem_base + buf * TT, da + 2u * kk, db + 2u * kk, idesc, in_group == 0 ? 0u : 1u);
+                    if (leader) {
+                        if (F8) umma_e4m3(tmem_base + buf * TT, da + 2u * kk, db + 2u * kk, idesc, in_group == 0 ? 0u : 1u);
+                        else    umma_i8(tmem_base + buf * TT, da + 2u * kk, db + 2u * kk, idesc, in_group == 0 ? 0u : 1u);
+                    }
                     if (++in_group == mma_per_group) {
                         if (leader) umma_commit(acc_full(buf));
                         in_group = 0;
@@ -370,10 +399,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                     const int row = idx >> 2, ch = idx & 3;
                     const uint4 pk = cur[i];
                     uint4 lo, hi;
-                    lo.x = (pk.x << 4) & 0xF0F0F0F0u; hi.x = pk.x & 0xF0F0F0F0u;
-                    lo.y = (pk.y << 4) & 0xF0F0F0F0u; hi.y = pk.y & 0xF0F0F0F0u;
-                    lo.z = (pk.z << 4) & 0xF0F0F0F0u; hi.z = pk.z & 0xF0F0F0F0u;
-                    lo.w = (pk.w << 4) & 0xF0F0F0F0u; hi.w = pk.w & 0xF0F0F0F0u;
+                    unpack32<F8>(pk, lo, hi);
                     const uint32_t drow = dst + (row >> 3) * 1024 + (row & 7) * 128;
                     sts128(drow + (((2 * ch) ^ (row & 7)) << 4), lo);
                     sts128(drow + (((2 * ch + 1) ^ (row & 7)) << 4), hi);
@@ -416,10 +442,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                             const int row = idx >> 2, ch = idx & 3;
                             const uint4 pk = cur[i];
                             uint4 lo, hi;
-                            lo.x = (pk.x << 4) & 0xF0F0F0F0u; hi.x = pk.x & 0xF0F0F0F0u;
-                            lo.y = (pk.y << 4) & 0xF0F0F0F0u; hi.y = pk.y & 0xF0F0F0F0u;
-                            lo.z = (pk.z << 4) & 0xF0F0F0F0u; hi.z = pk.z & 0xF0F0F0F0u;
-                            lo.w = (pk.w << 4) & 0xF0F0F0F0u; hi.w = pk.w & 0xF0F0F0F0u;
+                            unpack32<F8>(pk, lo, hi);
                             const uint32_t drow = dst + (row >> 3) * 1024 + (row & 7) * 128;
                             sts128(drow + (((2 * ch) ^ (row & 7)) << 4), lo);
                             sts128(drow + (((2 * ch + 1) ^ (row & 7)) << 4), hi);
@@ -448,6 +471,11 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         float acc[EC];
 #pragma unroll
         for (int j = 0; j < EC; ++j) acc[j] = 0.0f;
+        // E4M3 path: the operands are the integers themselves (no factor 16 to undo) and the accumulators
+        // arrive as fp32 holding exact integers, so a group costs one FMA per element and no conversion.
+        // (Packed two-lane FMAs measured the same: the drain is bound by the FMA pipe and the register
+        // file's write port, which the TMEM loads share, not by issue slots.)
+        const float sc_mul = F8 ? 16.0f : 1.0f;
         bool ok = true;
         // Scales are fetched two groups ahead with volatile loads: a plain load would be sunk next to
         // its use and expose the L2 latency once per group.
@@ -481,11 +509,17 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 tmem_wait_ld();
 #pragma unroll
                 for (int u = 0; u < GU; ++u) {
-                    float f[CH];
+                    if (F8) {
+                        const float s16 = scu[u] * sc_mul;
 #pragma unroll
-                    for (int j = 0; j < CH; ++j) asm volatile("cvt.rn.f32.s32 %0, %1;" : "=f"(f[j]) : "r"(c[u][j]));
+                        for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[j]) : "f"(__uint_as_float(c[u][j])), "f"(s16));
+                    } else {
+                        float f[CH];
 #pragma unroll
-                    for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[j]) : "f"(f[j]), "f"(scu[u]));
+                        for (int j = 0; j < CH; ++j) asm volatile("cvt.rn.f32.s32 %0, %1;" : "=f"(f[j]) : "r"(c[u][j]));
+#pragma unroll
+                        for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[j]) : "f"(f[j]), "f"(scu[u]));
+                    }
                 }
                 tcgen05_fence_before_sync();
                 __syncwarp();
@@ -502,7 +536,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             }
         }
         for (; g < n_groups && ok; ++g) {
-            const float sc = n_ok ? sc_next : 0.0f;
+            const float sc = n_ok ? sc_next * sc_mul : 0.0f;
             sc_next = sc_next2;
             if (g + 2 < n_groups) sc_next2 = ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + 2) * p.N);
             // lane 0 polls, the others wait at the shuffle: no 32-way spin, and the verdict is warp-uniform
@@ -524,11 +558,16 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 const uint32_t (&cur)[CH] = (ch & 1) ? c1 : c0;
                 // Convert the whole chunk first, then accumulate: every FMA then finds its operand ready
                 // instead of waiting out the conversion latency element by element.
-                float f[CH];
+                if (F8) {
 #pragma unroll
-                for (int j = 0; j < CH; ++j) asm volatile("cvt.rn.f32.s32 %0, %1;" : "=f"(f[j]) : "r"(cur[j]));
+                    for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[ch * CH + j]) : "f"(__uint_as_float(cur[j])), "f"(sc));
+                } else {
+                    float f[CH];
 #pragma unroll
-                for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[ch * CH + j]) : "f"(f[j]), "f"(sc));
+                    for (int j = 0; j < CH; ++j) asm volatile("cvt.rn.f32.s32 %0, %1;" : "=f"(f[j]) : "r"(cur[j]));
+#pragma unroll
+                    for (int j = 0; j < CH; ++j) asm volatile("fma.rn.f32 %0, %1, %2, %0;" : "+f"(acc[ch * CH + j]) : "f"(f[j]), "f"(sc));
+                }
                 if (DUMP) {
                     const int cc = n - p.aux.dump.col0;
                     if (p.aux.dump.acc != nullptr && n_ok && cc >= 0 && cc < p.aux.dump.cols) {
@@ -537,7 +576,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                             const int tok = m0 + h * EC + ch * CH + j;
                             const int rr = tok - p.aux.dump.row0;
                             if (tok < p.M && rr >= 0 && rr < p.aux.dump.rows)
-                                p.aux.dump.acc[(static_cast<size_t>(g0 + g) * p.aux.dump.rows + rr) * p.aux.dump.cols + cc] = static_cast<int>(cur[j]) >> 4;
+                                p.aux.dump.acc[(static_cast<size_t>(g0 + g) * p.aux.dump.rows + rr) * p.aux.dump.cols + cc] = F8 ? static_cast<int>(__uint_as_float(cur[j])) : static_cast<int>(cur[j]) >> 4;
                         }
                     }
                 }
@@ -655,7 +694,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 
 }  // namespace
 
-template <int TT, bool DUMP>
+template <int TT, bool DUMP, bool F8>
 static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaStream_t st)
 {
     using T = Tile<TT>;
@@ -686,7 +725,7 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = plan.pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_kernel<TT, DUMP>, a.tm_x, a.tm_y, p);
+    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_kernel<TT, DUMP, F8>, a.tm_x, a.tm_y, p);
 }
 
 // Tile and split choice.  Large M: 256-token tiles, no split.  M <= 256: the smallest tile that holds
@@ -729,8 +768,10 @@ size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_of
 cudaError_t gemm_i8_init()
 {
     cudaError_t e;
-#define RUDDER_I8_ATTR(TT, D)                                                                                          \
-    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT>::DYN_SMEM); \
+#define RUDDER_I8_ATTR(TT, D)                                                                                                 \
+    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT>::DYN_SMEM); \
+    if (e != cudaSuccess) return e;                                                                                           \
+    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT>::DYN_SMEM);  \
     if (e != cudaSuccess) return e;
     RUDDER_I8_ATTR(32, false) RUDDER_I8_ATTR(64, false) RUDDER_I8_ATTR(256, false)
     RUDDER_I8_ATTR(32, true) RUDDER_I8_ATTR(64, true) RUDDER_I8_ATTR(256, true)
@@ -742,11 +783,15 @@ cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st)
 {
     const GemmI8Plan plan = gemm_i8_plan(a.M, a.N, a.K, a.acc != nullptr);
     const bool dump = a.acc != nullptr;
+#define RUDDER_I8_LAUNCH(TT)                                                                                     \
+    return a.f8 ? (dump ? launch_one<TT, true, true>(a, plan, st) : launch_one<TT, false, true>(a, plan, st))   \
+                : (dump ? launch_one<TT, true, false>(a, plan, st) : launch_one<TT, false, false>(a, plan, st));
     switch (plan.token_tile) {
-        case 32:  return dump ? launch_one<32, true>(a, plan, st) : launch_one<32, false>(a, plan, st);
-        case 64:  return dump ? launch_one<64, true>(a, plan, st) : launch_one<64, false>(a, plan, st);
-        default:  return dump ? launch_one<256, true>(a, plan, st) : launch_one<256, false>(a, plan, st);
+        case 32:  RUDDER_I8_LAUNCH(32)
+        case 64:  RUDDER_I8_LAUNCH(64)
+        default:  RUDDER_I8_LAUNCH(256)
     }
+#undef RUDDER_I8_LAUNCH
 }
 
 }  // namespace rudder

@@ -36,6 +36,7 @@ struct SegParams {
 struct rudder_weight {
     int N, K, G, scheme;
     int device;
+    int f8;                   // W4A4 with groups up to 128: codes in the sign-magnitude layout, GEMM on the E4M3 tensor path
     uint8_t* codes;
     float* scales_t;
     void* scales_c;
@@ -63,12 +64,13 @@ struct ActqArgs {
 
 // ---- launches (each returns cudaGetLastError of its launch) ----------------------------------
 cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G, uint8_t* codes_il,
-                             float* scales_t, uint16_t* scales_c, float* dinv, int8_t* tmp_codes,
+                             float* scales_t, uint16_t* scales_c, float* dinv, int8_t* tmp_codes, bool signmag,
                              cudaStream_t st);
-cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, cudaStream_t st);
+cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, bool signmag, cudaStream_t st);
 
 cudaError_t actq_init();
-cudaError_t launch_actq_int(const ActqArgs& a, int qmax, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);
+// e4m3: the codes (integers in [-7, 7]) are written as E4M3 bytes for the FP8 tensor path instead of int8
+cudaError_t launch_actq_int(const ActqArgs& a, int qmax, bool e4m3, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);
 cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st);
 cudaError_t launch_pack_nvfp4(const float* W, const float* d, int N, int K, uint8_t* codes, uint8_t* sb_canonical,
                               uint8_t* sf_tiled, size_t sf_tiled_bytes, float* dinv, float* tensor_scale,
@@ -102,6 +104,7 @@ struct GemmI8Args {
     CUtensorMap tm_y;           // output bf16 [M, N] (row pitch ldy), box {min(128, N) channels, token tile}
     uint16_t* y;                // the same output as a plain pointer (small tiles are stored without TMA)
     int64_t ldy;
+    bool f8;                    // E4M3 operands (exact small integers), FP32 accumulators
     const CUtensorMap* tm_w;    // device-resident tensor map over the packed weights (256-token tiles stage them by TMA)
     const uint8_t* w_codes;     // packed INT4 weights
     const float* w_scales_t;    // [K/G][N]

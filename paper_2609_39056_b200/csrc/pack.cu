@@ -61,6 +61,57 @@ __global__ void pack_int4_interleave_kernel(const int8_t* __restrict__ q, int N,
     codes_il[idx] = static_cast<uint8_t>((lo & 0xF) | ((hi & 0xF) << 4));
 }
 
+// Layout for the FP8 tensor path (W4A4 with group scales): sign and magnitude apart, arranged so that the
+// GEMM's unpack turns one 32-bit word into eight E4M3 bytes with two byte-permute look-ups.  Word j of
+// the 16-byte piece c covers channels A_i = 32 c + 4 j + i and B_i = 32 c + 16 + 4 j + i (i = 0..3):
+//   bits [4i, 4i+3)       |A_i|        bits [16+4i, 16+4i+3)   |B_i|
+//   bit 3 + 8i            sign of A_i  bit 7 + 8i              sign of B_i
+// (every sign sits in bit 3 of some nibble, which the look-up's selector masks away).
+__device__ __forceinline__ uint32_t sm_word(const int8_t* qa, const int8_t* qb)
+{
+    uint32_t w = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int a = qa[i], b = qb[i];
+        w |= static_cast<uint32_t>(a < 0 ? -a : a) << (4 * i);
+        w |= static_cast<uint32_t>(b < 0 ? -b : b) << (16 + 4 * i);
+        w |= static_cast<uint32_t>(a < 0) << (3 + 8 * i);
+        w |= static_cast<uint32_t>(b < 0) << (7 + 8 * i);
+    }
+    return w;
+}
+__global__ void pack_int4_signmag_kernel(const int8_t* __restrict__ q, int N, int K, uint32_t* __restrict__ codes_sm)
+{
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;      // one 32-bit word
+    const size_t total = static_cast<size_t>(N) * (K / 8);
+    if (idx >= total) return;
+    const size_t n = idx / (K / 8);
+    const int word = static_cast<int>(idx % (K / 8));
+    const int c = word >> 2, j = word & 3;
+    const int8_t* base = q + n * K + 32 * c + 4 * j;
+    codes_sm[idx] = sm_word(base, base + 16);
+}
+__global__ void export_int4_signmag_kernel(const uint32_t* __restrict__ codes_sm, int N, int K, uint8_t* __restrict__ out)
+{
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const size_t total = static_cast<size_t>(N) * (K / 2);
+    if (idx >= total) return;
+    const size_t n = idx / (K / 2);
+    const int k0 = static_cast<int>(idx % (K / 2)) * 2;
+    uint8_t nib[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int k = k0 + t;
+        const int c = k >> 5, p = k & 31;
+        const int is_b = p >> 4, j = (p & 15) >> 2, i = p & 3;
+        const uint32_t w = codes_sm[n * (K / 8) + 4 * c + j];
+        const int mag = static_cast<int>((w >> (16 * is_b + 4 * i)) & 7u);
+        const int neg = static_cast<int>((w >> ((is_b ? 7 : 3) + 8 * i)) & 1u);
+        nib[t] = static_cast<uint8_t>((neg ? -mag : mag) & 0xF);
+    }
+    out[idx] = static_cast<uint8_t>(nib[0] | (nib[1] << 4));
+}
+
 __global__ void dinv_kernel(const float* __restrict__ d, int K, float* __restrict__ dinv)
 {
     const int k = blockIdx.x * blockDim.x + threadIdx.x;
@@ -87,7 +138,7 @@ __global__ void export_int4_kernel(const uint8_t* __restrict__ codes_il, int N, 
 }
 
 cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G, uint8_t* codes_il,
-                             float* scales_t, uint16_t* scales_c, float* dinv, int8_t* tmp_codes,
+                             float* scales_t, uint16_t* scales_c, float* dinv, int8_t* tmp_codes, bool signmag,
                              cudaStream_t st)
 {
     const long long warps = static_cast<long long>(N) * (K / G);
@@ -97,16 +148,22 @@ cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t total = static_cast<size_t>(N) * (K / 2);
-    pack_int4_interleave_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(tmp_codes, N, K, codes_il);
+    if (signmag)
+        pack_int4_signmag_kernel<<<static_cast<unsigned>((total / 4 + 255) / 256), 256, 0, st>>>(tmp_codes, N, K, reinterpret_cast<uint32_t*>(codes_il));
+    else
+        pack_int4_interleave_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(tmp_codes, N, K, codes_il);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     dinv_kernel<<<(K + 255) / 256, 256, 0, st>>>(d, K, dinv);
     return cudaGetLastError();
 }
 
-cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, cudaStream_t st)
+cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, bool signmag, cudaStream_t st)
 {
     const size_t total = static_cast<size_t>(N) * (K / 2);
+    if (signmag)
+        export_int4_signmag_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(reinterpret_cast<const uint32_t*>(codes_il), N, K, canonical);
+    else
     export_int4_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(codes_il, N, K, canonical);
     return cudaGetLastError();
 }

@@ -201,6 +201,26 @@ __device__ __forceinline__ uint32_t umma_idesc_i8(int m, int n) {
     return d;
 }
 
+// Instruction descriptor for kind::f8f6f4 with E4M3 A and B, both K-major, FP32 accumulate.
+__device__ __forceinline__ uint32_t umma_idesc_e4m3(int m, int n) {
+    uint32_t d = 0;
+    d |= 1u << 4;                 // D format: F32   (A and B formats: 0 = E4M3)
+    d |= static_cast<uint32_t>(n >> 3) << 17;
+    d |= static_cast<uint32_t>(m >> 4) << 24;
+    return d;
+}
+__device__ __forceinline__ void umma_e4m3(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t"
+        "}\n"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // D[tmem] (+)= A[smem] * B[smem]^T, one CTA, issued by a single thread.
 __device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
                                         uint32_t accumulate) {

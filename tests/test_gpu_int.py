@@ -24,11 +24,12 @@ def _assert_clean(rd):
     assert last == 0, f"device status {last} (wait code {where})"
 
 
+@pytest.mark.parametrize("scheme", ["w4a8", "w4a4"])       # w4a4 with G <= 128 is stored in its own (sign-magnitude) layout
 @pytest.mark.parametrize("N,K,G", [(64, 128, 64), (128, 256, 128), (256, 512, 512), (320, 1024, 64)])
-def test_pack_export_bit_exact(rd, N, K, G):
+def test_pack_export_bit_exact(rd, N, K, G, scheme):
     inp = wl.tiny(seed=100 + N, M=4, K=K, N=N)
     ref = oracle.pack_int4(inp.W, inp.d, G)
-    g = GpuLinear(rd, inp, "w4a8", G)
+    g = GpuLinear(rd, inp, scheme, G)
     ex = rd.rudder_weight_export(g.w)
     assert np.array_equal(ex["codes"].cpu().numpy(), ref["packed"])
     assert np.array_equal(ex["scales"].view(torch.int16).cpu().numpy().view(np.uint16), ref["scales"])
@@ -57,10 +58,11 @@ def test_pack_degenerate_weights(rd):
     inp.W[11, 0:64] = np.tile(np.array([7.0, 3.5, 2.5, 1.5, 0.5, -0.5, -2.5, -6.5], np.float32), 8) * 0.01
     inp.d[:] = 1.0
     ref = oracle.pack_int4(inp.W, inp.d, 64)
-    g = GpuLinear(rd, inp, "w4a8", 64)
-    ex = rd.rudder_weight_export(g.w)
-    assert np.array_equal(ex["scales"].cpu().numpy().view(np.uint16), ref["scales"].view(np.uint16))
-    assert np.array_equal(ex["codes"].cpu().numpy(), ref["packed"])
+    for scheme in ("w4a8", "w4a4"):
+        g = GpuLinear(rd, inp, scheme, 64)
+        ex = rd.rudder_weight_export(g.w)
+        assert np.array_equal(ex["scales"].cpu().numpy().view(np.uint16), ref["scales"].view(np.uint16))
+        assert np.array_equal(ex["codes"].cpu().numpy(), ref["packed"])
     _assert_clean(rd)
 
 
@@ -105,6 +107,10 @@ CASES = [
     (257, 1024, 512, 64, "w4a4"),
     (96, 256, 256, 128, "w4a4"),
     (33, 2304, 256, 64, "w4a8"),       # 18 stages: every ring wraps several times
+    (20, 512, 320, 64, "w4a4"),        # W4A4 with group scales runs on the E4M3 tensor path: 32-token tiles, ragged N
+    (200, 2304, 256, 128, "w4a4"),     # 64-token tiles, 18 stages
+    (300, 640, 128, 64, "w4a4"),       # 256-token tiles with a ragged tail
+    (64, 512, 256, 512, "w4a4"),       # G = K stays on the integer path
 ]
 
 
@@ -127,6 +133,34 @@ def test_linear_accumulators_and_output(rd, M, K, N, G, scheme, mode):
     # the production entry point (no dump) gives the same bits
     Y2 = rd.rudder_linear(g.w, g.X, g.seg, step, g.tab, g.bias)
     assert torch.equal(Y, Y2)
+    _assert_clean(rd)
+
+
+@pytest.mark.parametrize("G", [64, 128])
+@pytest.mark.parametrize("M", [40, 300])
+def test_w4a4_extreme_sums_are_exact(rd, G, M):
+    """Every code at +-7: the group sums reach +-49 G, the largest magnitude the E4M3 / FP32-accumulator
+    path has to hold exactly.  Row 0 and channel 0 are all-positive (sum = 49 G), the rest random signs."""
+    K, N = 512, 128
+    inp = wl.tiny(seed=977 + G + M, M=M, K=K, N=N)
+    rng = np.random.default_rng(5)
+    sw = rng.choice(np.array([-1.0, 1.0], np.float32), size=(N, K)); sw[0, :] = 1.0
+    sx = rng.choice(np.array([-1.0, 1.0], np.float32), size=(M, K)); sx[0, :] = 1.0; sx[1, :] = -1.0
+    inp.W[:] = 0.03 * sw
+    inp.d[:] = 1.0
+    X = (2.0 * sx).astype(np.float32)
+    inp.X_bf16[:] = (X.view(np.uint32) >> 16).astype(np.uint16)        # +-2.0 is exact in bf16
+    ref_w = oracle.pack_int4(inp.W, inp.d, G)
+    assert np.all(np.abs(ref_w["qw"]) == 7)
+    g = GpuLinear(rd, inp, "w4a4", G)
+    Y, acc = rd.rudder_linear_dump_acc(g.w, g.X, g.seg, 0, g.tab, g.bias)
+    rc, rr = oracle.quantize_int(inp.X_bf16, ref_w["dinv"], inp.gamma, None, 0, 0, inp.seg_offsets, inp.seg_stream, 7)
+    assert np.all(np.abs(rc) == 7)
+    racc = oracle.accumulate_int(rc, ref_w["qw"], G)
+    assert racc[0, 0, 0] == 49 * G and racc[0, 1, 0] == -49 * G
+    assert np.array_equal(acc.cpu().numpy(), racc)
+    _, y64 = oracle.linear_int(rc, rr, ref_w["qw"], ref_w["scales"], G, inp.bias)
+    check_output(bf16_to_np(Y), y64)
     _assert_clean(rd)
 
 
