@@ -231,10 +231,35 @@ def roofline_of(cfg, m, pk):
             "per_kernel_ms": [float(v) for v in m["prof"]]}
 
 
-def small_m_sweep(rd, torch, dev, pk, schemes=("w4a8", "w4a4"), sizes=(2048, 4096), rows=(16, 64, 128, 256)):
-    """Configuration 4: action + proprio-only passes; one packed weight reused across 20 steps, captured
-    in one CUDA graph (weights stay L2-resident: `algorithmic` GB/s counts every byte the call must move)."""
+def _graph_us(torch, stream, calls):
+    """Median device time (us) per call of a CUDA graph holding `calls` (a list of closures), 5 warm-up + 20 timed replays."""
+    with torch.cuda.stream(stream):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for c in calls:
+                c()
+        for _ in range(5):
+            graph.replay()
+        stream.synchronize()
+        times = []
+        for _ in range(20):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            graph.replay()
+            e1.record(stream)
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1) / len(calls))
+    return float(np.median(times)) * 1e3
+
+
+def small_m_sweep(rd, torch, dev, pk, schemes=("w4a8", "w4a4"), sizes=(2048, 4096), rows=(16, 64, 128, 256), cold=True):
+    """Configuration 4: action + proprio-only passes.  (i) One packed weight reused across 20 steps, captured
+    in one CUDA graph (weights stay L2-resident: `algorithmic` GB/s counts every byte the call must move).
+    (ii) `cold`: the same call over a rotation of distinct packed weights whose total size is several
+    times the L2 (at least 64 of them), one graph of one linear per weight: every weight comes from HBM,
+    as in a model whose layers do not fit the cache."""
     out = []
+    L2_BYTES = 126e6
     for scheme in schemes:
         for KN in sizes:
             for M in rows:
@@ -254,26 +279,24 @@ def small_m_sweep(rd, torch, dev, pk, schemes=("w4a8", "w4a4"), sizes=(2048, 409
                     for t in range(3):
                         rd.rudder_linear(w, X, seg, t, tab, bias, Y=Y, workspace=ws)
                     stream.synchronize()
-                    graph = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(graph, stream=stream):
-                        for t in range(cfg.T):
-                            rd.rudder_linear(w, X, seg, t, tab, bias, Y=Y, workspace=ws)
-                    for _ in range(5):
-                        graph.replay()
-                    stream.synchronize()
-                    times = []
-                    for _ in range(20):
-                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                        e0.record(stream)
-                        graph.replay()
-                        e1.record(stream)
-                        e1.synchronize()
-                        times.append(e0.elapsed_time(e1) / cfg.T)
-                us = float(np.median(times)) * 1e3
+                us = _graph_us(torch, stream, [
+                    (lambda t=t: rd.rudder_linear(w, X, seg, t, tab, bias, Y=Y, workspace=ws)) for t in range(cfg.T)])
                 nbytes = algorithmic_bytes_linear(M, KN, KN, cfg.group, scheme)
-                out.append({"scheme": scheme, "M": M, "K": KN, "N": KN, "us_per_linear": us,
-                            "algorithmic_gbs": nbytes / (us * 1e-6) / 1e9, "hbm_frac": nbytes / (us * 1e-6) / 1e9 / pk["hbm_gbs"],
-                            "tops": 2.0 * M * KN * KN / (us * 1e-6) / 1e12})
+                row = {"scheme": scheme, "M": M, "K": KN, "N": KN, "us_per_linear": us,
+                       "algorithmic_gbs": nbytes / (us * 1e-6) / 1e9, "hbm_frac": nbytes / (us * 1e-6) / 1e9 / pk["hbm_gbs"],
+                       "tops": 2.0 * M * KN * KN / (us * 1e-6) / 1e12}
+                if cold:
+                    w_bytes = KN * KN // 2 + (KN // cfg.group) * KN * 6        # codes + fp32 and fp16 scale copies
+                    n_w = max(64, int(np.ceil(3 * L2_BYTES / w_bytes)))
+                    rotation = [w] + [rd.rudder_pack_weights(W, d, rd.SCHEMES[scheme], cfg.group) for _ in range(n_w - 1)]
+                    us_c = _graph_us(torch, stream, [
+                        (lambda i=i: rd.rudder_linear(rotation[i], X, seg, i % cfg.T, tab, bias, Y=Y, workspace=ws))
+                        for i in range(n_w)])
+                    row.update({"cold_weights": n_w, "us_per_linear_cold": us_c,
+                                "algorithmic_gbs_cold": nbytes / (us_c * 1e-6) / 1e9,
+                                "hbm_frac_cold": nbytes / (us_c * 1e-6) / 1e9 / pk["hbm_gbs"]})
+                    del rotation
+                out.append(row)
                 del w
     return out
 

@@ -51,7 +51,9 @@ typedef enum {
 /* Activation / weight number formats.  Weights are always 4-bit. */
 typedef enum {
     RUDDER_W4A8_INT = 0,    /* INT4 weights (group scales), INT8 activations, q_max = 127 (Eq. 1, k = 8) */
-    RUDDER_W4A4_INT = 1,    /* INT4 weights, INT4 activations, q_max = 7 (Eq. 1, k = 4), int8 tensor-core path */
+    RUDDER_W4A4_INT = 1,    /* INT4 weights, INT4 activations, q_max = 7 (Eq. 1, k = 4); 8-bit tensor-core path
+                               (integer MMA, or its exact E4M3 / FP32-accumulator form when group <= 128:
+                               same integers, same results) */
     RUDDER_W4A4_NVFP4 = 2   /* E2M1 codes with a UE4M3 scale per 16 elements and an fp32 outer scale */
 } rudder_scheme;
 

@@ -7,7 +7,15 @@
 // thread) therefore owns one output channel, so the weight scale Delta_W[j,g] of a group is a single
 // register per thread and the per-group drain is exactly one int->float conversion and one FMA per
 // element.  That drain, not the tensor core, bounds the group-scaled path: the conversion pipe
-// sustains about 64 elements per clock per SM against 128 for the MMA at G = 64.
+// sustains about 64 elements per clock per SM against 128 for the MMA at G = 64, and every value
+// drained costs register-file writes (TMEM load, conversion, FMA) on the same four sub-partitions.
+//
+// W4A4 with group scales (G <= 128) takes the E4M3 form of the same product: codes in [-7, 7] are
+// exact in E4M3, |C^(g)| <= 128 * 49 is exact in the FP32 accumulators of kind::f8f6f4 (same tensor
+// rate as kind::i8), so C^(g) arrives as fp32 and the drain is the FMA alone.  The activations come
+// from the prologue as E4M3 bytes, the weights are stored sign-magnitude so that the unpack is two
+// table look-ups (byte permutes) per eight weights.  The integers, and therefore the results, are
+// the same bit for bit as on the INT32 path.
 //
 // Warp roles (warpgroup-aligned so that registers can be moved between them):
 //   warp 0        TMA producer: activation codes (int8 [TT tokens][128 B], 128-byte swizzle)
@@ -88,7 +96,7 @@ template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256, 6
 
 struct Params {
     int M, N, K, G;
-    const uint8_t* codes;        // packed INT4 weights [N][K/2], 32-channel interleave
+    const uint8_t* codes;        // packed INT4 weights [N][K/2], 32-channel interleave (E4M3 path: sign-magnitude words)
     const float* scales_t;       // [K/G][N] fp32 = Delta_W / 16
     const float* row_scale;      // r [M]
     const float* bias;           // [N] or nullptr
@@ -494,12 +502,10 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 float scu[GU];
 #pragma unroll
                 for (int u = 0; u < GU; ++u) scu[u] = n_ok ? ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + u) * p.N) : 0.0f;
-                if (lane == 0) {
 #pragma unroll
-                    for (int u = 0; u < GU; ++u)
-                        ok = ok && mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf + u), phb, abortp, W_ACC_FULL);
-                }
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                for (int u = 0; u < GU; ++u)
+                    ok = ok && mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf + u), phb, abortp, W_ACC_FULL);
+                ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 tcgen05_fence_after_sync();
                 uint32_t c[GU][CH];
@@ -539,10 +545,10 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             const float sc = n_ok ? sc_next * sc_mul : 0.0f;
             sc_next = sc_next2;
             if (g + 2 < n_groups) sc_next2 = ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + 2) * p.N);
-            // lane 0 polls, the others wait at the shuffle: no 32-way spin, and the verdict is warp-uniform
-            // (the TMEM loads below are warp-collective)
-            if (lane == 0) ok = mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), phb, abortp, W_ACC_FULL);
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            // the verdict is made warp-uniform (the TMEM loads below are warp-collective)
+            // every lane polls: a single polling lane followed by a shuffle measured 10 % slower per group
+            ok = mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), phb, abortp, W_ACC_FULL);
+            ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tcgen05_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + buf * TT + h * EC;
