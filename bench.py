@@ -150,9 +150,10 @@ def build_block(rd, cfg, torch, dev):
 # ncu capture of that launch; summaries under profiles/).  Keyed by workload; None = not captured.
 NCU_TRAFFIC_BYTES = {
     # sum over the kernel's 4 launches of one step (profiles/gemm_nvfp4_and_actq_cfg3_metrics.md,
-    # profiles/gemm_i8_w4_and_actq_cfg2_metrics.md)
+    # profiles/gemm_i8_w4_and_actq_cfg2_metrics.md, profiles/gemm_i8_w4_f8_and_actq_cfg3_w4a4_metrics.md)
     "cfg3_nvfp4_block_h3072_f12288_m17536": 1287.4e6,
-    "cfg2_w4a8_block_h2048_f8192_m4416": 123.4e6,
+    "cfg2_w4a8_block_h2048_f8192_m4416": 119.2e6,
+    "cfg3_w4a4_block_h3072_f12288_m17536": 1791.5e6,
 }
 
 
