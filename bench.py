@@ -9,7 +9,7 @@ action) tokens, 10 steps of tables).  The W4A8 block (configuration 2), the W4A4
 (configuration 3) and the small-M sweep (configuration 4) are measured in the same run and reported
 under "also" (rank 0, N = 1).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg2_g128|cfg2_perchannel|cfg3|cfg3_nvfp4|cfg4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg2_g128|cfg2_perchannel|cfg2_perchannel_static|cfg3|cfg3_nvfp4|cfg4] [--impl reference]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded row sample.
 """
@@ -52,11 +52,14 @@ def workload_config(name: str):
         return wl.config(3, "w4a4")
     if name == "cfg3_nvfp4":
         return wl.config(3, "nvfp4")
-    if name in ("cfg2_g128", "cfg2_perchannel"):      # configuration 2 at the other weight-scale granularities
+    if name in ("cfg2_g128", "cfg2_perchannel", "cfg2_perchannel_static"):      # configuration 2 at the other granularities
         import dataclasses
         c = wl.config(2)
         g = 128 if name == "cfg2_g128" else 0         # 0: one scale per output channel (Eq. 10 as printed)
-        return dataclasses.replace(c, name=c.name + ("_g128" if g else "_per_channel"), group=g)
+        # "_static": one calibrated threshold per step for all rows, the activation setting of the
+        # paper's sensitivity study (per-output-channel W4, static per-tensor A8)
+        suffix = "_g128" if g else ("_per_channel_static" if name.endswith("_static") else "_per_channel")
+        return dataclasses.replace(c, name=c.name + suffix, group=g)
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -138,7 +141,18 @@ def build_block(rd, cfg, torch, dev):
         ws.append(rd.rudder_pack_weights(W, d, scheme, cfg.group or l.K))     # group 0: one scale per output channel (G = K)
         del W, d
         gamma = torch.from_numpy(l.gamma).to(dev)
-        tabs.append(rd.ScaleTable(gamma, None, rd.RANGE_PER_TOKEN))
+        if cfg.name.endswith("_static"):
+            # input recipe, step 8: clip[t] = 99.9th percentile of |(x dinv) gamma[t, s(i)]| over all rows
+            x = torch.from_numpy(l.X_bf16.view(np.int16)).to(dev).view(torch.bfloat16).float()
+            x *= rd.rudder_weight_export(ws[-1])["dinv"][None, :]
+            row_stream = torch.from_numpy(np.repeat(l.seg_stream, np.diff(l.seg_offsets)).astype(np.int64)).to(dev)
+            k = max(1, int(round(0.999 * x.numel())))
+            clip = torch.stack([torch.kthvalue((x * gamma[t][row_stream][:, None]).abs().flatten(), k).values
+                                for t in range(gamma.shape[0])]).float().contiguous()
+            del x
+            tabs.append(rd.ScaleTable(gamma, clip, rd.RANGE_STATIC))
+        else:
+            tabs.append(rd.ScaleTable(gamma, None, rd.RANGE_PER_TOKEN))
         biases.append(torch.from_numpy(l.bias).to(dev))
         xs.append(torch.from_numpy(l.X_bf16.view(np.int16)).to(dev).view(torch.bfloat16))
         ys.append(torch.empty((l.M, l.N), dtype=torch.bfloat16, device=dev))
@@ -407,7 +421,7 @@ def run_ours(args):
         del m, ws, tabs, biases, xs, ys, workspace, lins
         torch.cuda.empty_cache()
         also = {}
-        for name in ("cfg2", "cfg2_g128", "cfg2_perchannel", "cfg3", "cfg3_nvfp4"):
+        for name in ("cfg2", "cfg2_g128", "cfg2_perchannel", "cfg2_perchannel_static", "cfg3", "cfg3_nvfp4"):
             if name == args.workload:
                 continue
             c2 = workload_config(name)
@@ -429,7 +443,7 @@ def run_ours(args):
                                                               "nvfp4": "e2m1 x e2m1 (ue4m3 block scales) -> fp32"}[cfg.scheme],
             "data": "synthetic", "gpu_launches": 8 * args.steps,
             "config": {"workload": cfg.name, "scheme": cfg.scheme, "group": 16 if cfg.scheme == "nvfp4" else cfg.group, "M": M,
-                       "linears": {n: [K, N] for n, K, N in cfg.linears}, "range_mode": "per_token",
+                       "linears": {n: [K, N] for n, K, N in cfg.linears}, "range_mode": "static" if cfg.name.endswith("_static") else "per_token",
                        "steps_of_tables": T, "tops_per_step": ops / 1e12,
                        "l2": f"working set per step {sum(alg_bytes) / 1e6:.0f} MB (inputs {sum(2 * M * K for _, K, _ in cfg.linears) / 1e6:.0f} MB) exceeds the 126 MB L2; no explicit flush",
                        "parallelism": f"replicas x{world} (rows independent, no collective)"},
@@ -457,12 +471,24 @@ def cpu_baseline(cfg, lins, target_s=15.0, impl_reference=False):
     for l in lins:
         packs.append(oracle.pack_nvfp4(l.W, l.d) if cfg.scheme == "nvfp4" else oracle.pack_int4(l.W, l.d, cfg.group or l.K))
     M = cfg.M
+    static = cfg.name.endswith("_static")
+    clips = []
+    for l, pw in zip(lins, packs):
+        if not static:
+            clips.append(None)
+            continue
+        # the workload's threshold (99.9th percentile of |(x dinv) gamma|), here from every 16th row: the
+        # oracle's time does not depend on its value
+        X = wl.bf16_bits_to_f32(l.X_bf16[::16])
+        st = np.repeat(l.seg_stream, np.diff(l.seg_offsets))[::16]
+        clips.append(np.array([np.percentile(np.abs((X * pw["dinv"][None, :]) * l.gamma[t, st][:, None]), 99.9)
+                               for t in range(l.gamma.shape[0])], np.float32))
 
     def run(rows):
         t0 = time.time()
-        for l, pw in zip(lins, packs):
-            oracle.rudder_linear(l.X_bf16, pw, l.gamma, None, 0, oracle.RANGE_PER_TOKEN, l.seg_offsets, l.seg_stream,
-                                 cfg.scheme, l.bias, rows=rows)
+        for l, pw, clip in zip(lins, packs, clips):
+            oracle.rudder_linear(l.X_bf16, pw, l.gamma, clip, 0, oracle.RANGE_STATIC if static else oracle.RANGE_PER_TOKEN,
+                                 l.seg_offsets, l.seg_stream, cfg.scheme, l.bias, rows=rows)
         return time.time() - t0
 
     rng = np.random.default_rng(1234)
