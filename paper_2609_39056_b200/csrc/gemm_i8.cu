@@ -46,6 +46,13 @@
 // order (deterministic) and stores its bf16 results straight from registers.  The kernel is launched
 // with programmatic dependent launch: everything that does not read the prologue's output (barrier
 // set-up, TMEM allocation) overlaps the prologue kernel.
+// Persistent form (256-token tiles, one scale per output channel, at least three tiles per SM): one CTA
+// per SM walks tiles blockIdx.x, + gridDim.x, ...  With a single weight group per tile the drain warps
+// are idle during the main loop, so the whole tail of a tile -- drain, scaling, staging, store -- runs
+// under the next tile's MMAs (the two TMEM buffers alternate per tile).  The output leaves through a
+// 32 KB slab of its own (128 tokens x 128 channels, half a tile at a time, one TMA store each, waited for
+// only when the slab is needed again); the rings give up one stage each to pay for it; the row scales
+// of the next tile are staged by the otherwise idle warp 2 through two shared-memory slots.
 // TMEM: NBUF = 512 / TT (at most 8) buffers of TT columns x 128 lanes of INT32, one weight group each.
 // acc_full[b]: umma commit; acc_empty[b]: 8 epilogue warps.
 #include "internal.cuh"
@@ -59,7 +66,15 @@ namespace {
 
 constexpr int BN = 128;          // output channels per tile (MMA M)
 constexpr int KSTAGE = 128;      // input channels (= bytes of int8 per row) per pipeline stage
-constexpr int SW = 4;            // unpacked-weight stages
+#ifndef RUDDER_PSX
+#define RUDDER_PSX 3             // persistent form: activation stages
+#endif
+#ifndef RUDDER_PSW
+#define RUDDER_PSW 3             // persistent form: unpacked-weight stages
+#endif
+#ifndef RUDDER_PERSIST_MIN_G
+#define RUDDER_PERSIST_MIN_G 0   // (build-time switch: a huge value turns the persistent form off)
+#endif
 constexpr int W_BYTES = BN * KSTAGE;
 constexpr int SR = 4;            // packed-weight stages (256-token tiles)
 constexpr int RAW_BYTES = BN * KSTAGE / 2;
@@ -77,21 +92,28 @@ constexpr int RUDDER_SLEEP_UNPACK = 64;
 constexpr int RUDDER_SLEEP_MMA = 0;
 constexpr int RUDDER_SLEEP_EPI = 0;
 
-template <int TT> struct Tile {          // TT = tokens per tile (MMA N): 256, 64 or 32
-    static constexpr int SX = (TT == 256) ? 4 : 8;
+// TT = tokens per tile (MMA N): 256, 64 or 32.  PERSIST (256 only): the CTA walks several tiles; a slab
+// of 128 tokens x 128 channels of bf16 output gets its own shared memory (the rings belong to the next
+// tile by the time a tile is written), paid for with shallower rings.
+template <int TT, bool PERSIST = false> struct Tile {
+    static constexpr int SX = PERSIST ? RUDDER_PSX : ((TT == 256) ? 4 : 8);
+    static constexpr int SW = PERSIST ? RUDDER_PSW : 4;  // unpacked-weight stages
     static constexpr int PD = (TT <= 64) ? 4 : 1;    // stages of packed weights a thread keeps in flight
     static constexpr int X_BYTES = TT * KSTAGE;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + SX * X_BYTES;
     static constexpr bool RAW = (TT == 256);         // packed weights staged by TMA (one more ring) instead of registers
     static constexpr int OFF_RAW = OFF_W + SW * W_BYTES;
-    static constexpr int BYTES = OFF_RAW + (RAW ? SR * RAW_BYTES : 0);
+    static constexpr int OFF_OUT = OFF_RAW + (RAW ? SR * RAW_BYTES : 0);
+    static constexpr int OUT_BYTES = 128 * BN * 2;   // persistent form: half a tile of bf16 results
+    static constexpr int BYTES = OFF_OUT + (PERSIST ? OUT_BYTES : 0);
     static constexpr int DYN_SMEM = BYTES + 1024;    // slack to align the base to 1024 bytes
     static constexpr int NBUF = (512 / TT > 8) ? 8 : 512 / TT;   // TMEM accumulator buffers (one weight group each)
     static constexpr int TMEM_COLS = NBUF * TT;
     static constexpr int EC = TT / 2;                // tokens per epilogue thread
     static constexpr int CH = (EC < 32) ? EC : 32;   // tokens per TMEM load
-    static_assert(SX * X_BYTES >= TT * BN * 2, "the output tile is staged over the X ring");
+    static_assert(PERSIST || SX * X_BYTES >= TT * BN * 2, "the output tile is staged over the X ring");
+    static_assert(!PERSIST || TT == 256, "the persistent form is built for 256-token tiles");
 };
 
 struct Params {
@@ -198,24 +220,33 @@ __device__ __forceinline__ void unpack32(const uint4& pk, uint4& lo, uint4& hi) 
     unpack8<F8>(pk.w, lo.w, hi.w);
 }
 
-template <int TT, bool DUMP, bool F8>
+template <int TT, bool DUMP, bool F8, bool PERSIST>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y, const Params p)
 {
-    using T = Tile<TT>;
+    using T = Tile<TT, PERSIST>;
+    constexpr int SW = T::SW;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * SW + 2 * T::NBUF + 1 + 2 * SR];
-    __shared__ __align__(16) float rs_smem[TT];      // row scales r_i of the tile's tokens (0 past M)
+    __shared__ __align__(8) uint64_t bars[2 * T::SX + 2 * T::SW + 2 * T::NBUF + 1 + 2 * SR + 4];
+    __shared__ __align__(16) float rs_smem[PERSIST ? 2 * TT : TT];   // row scales r_i of the tile's tokens (0 past M); persistent form: two tiles' worth
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_word;
     __shared__ int last_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    int tile_m, tile_n;
-    tile_coords(blockIdx.x, p.m_tiles, p.n_tiles, 16, tile_m, tile_n);
-    const int m0 = tile_m * TT;              // first token of the tile
-    const int n0 = tile_n * BN;              // first output channel of the tile
+    // PERSIST (256-token tiles, no K split): the CTA walks tiles blockIdx.x, + gridDim.x, ...; rings, TMEM
+    // buffers and their phases simply carry on from one tile to the next, so the MMAs of the next tile
+    // run while the drain warps scale, stage and store the current one.
+    // Otherwise the grid has one CTA per tile and every tile loop below runs once.
+    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int tile_step = PERSIST ? static_cast<int>(gridDim.x) : total_tiles;
+    auto tile_origin = [&](int tile, int& m0, int& n0) {
+        int tile_m, tile_n;
+        tile_coords(tile, p.m_tiles, p.n_tiles, 16, tile_m, tile_n);
+        m0 = tile_m * TT;                    // first token of the tile
+        n0 = tile_n * BN;                    // first output channel of the tile
+    };
     // this CTA's share of K: stages [s0, s0 + n_stages), weight groups [g0, g0 + n_groups)
     const int n_stages = p.stages_per_split;
     const int s0 = blockIdx.y * n_stages;
@@ -235,6 +266,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
     const uint32_t rs_full = bar0 + 8u * (2 * T::SX + 2 * SW + 2 * T::NBUF);
     auto raw_full = [&](int i) { return rs_full + 8u * (1 + i); };
     auto raw_empty = [&](int i) { return rs_full + 8u * (1 + SR + i); };
+    auto rsp_full = [&](int i) { return rs_full + 8u * (1 + 2 * SR + i); };        // persistent form: row-scale slots
+    auto rsp_empty = [&](int i) { return rs_full + 8u * (1 + 2 * SR + 2 + i); };
 
     if (threadIdx.x == 0) {
         abort_word = 0;
@@ -244,6 +277,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         mbar_init(rs_full, 1);
         if (T::RAW)
             for (int i = 0; i < SR; ++i) { mbar_init(raw_full(i), 1); mbar_init(raw_empty(i), UNPACK_THREADS / 32); }
+        if (PERSIST)
+            for (int i = 0; i < 2; ++i) { mbar_init(rsp_full(i), 1); mbar_init(rsp_empty(i), EPI_THREADS / 32); }
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -271,13 +306,17 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             bool ok = true;
             int slot = 0;
             uint32_t ph = 0;
-            for (int s = 0; s < n_stages; ++s) {
-                ok = mbar_wait<RUDDER_SLEEP_PROD>(x_empty(slot), ph ^ 1u, abortp, W_X_EMPTY);
-                if (!ok) break;
-                mbar_expect_tx(x_full(slot), p.x_tx);
-                tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, (s0 + s) * KSTAGE, m0, x_full(slot));
-                ++issued;
-                if (++slot == T::SX) { slot = 0; ph ^= 1u; }
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += tile_step) {
+                int m0, n0;
+                tile_origin(tile, m0, n0);
+                for (int s = 0; s < n_stages; ++s) {
+                    ok = mbar_wait<RUDDER_SLEEP_PROD>(x_empty(slot), ph ^ 1u, abortp, W_X_EMPTY);
+                    if (!ok) break;
+                    mbar_expect_tx(x_full(slot), p.x_tx);
+                    tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, (s0 + s) * KSTAGE, m0, x_full(slot));
+                    ++issued;
+                    if (++slot == T::SX) { slot = 0; ph ^= 1u; }
+                }
             }
             if (!ok) {
                 // Gave up: let the copies already in flight land before the CTA's shared memory goes away.
@@ -301,6 +340,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             int g_issued = 0;                          // groups started so far
             int sx = 0, sw = 0;                        // ring slots
             uint32_t phx = 0, phw = 0;                 // ring phases
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += tile_step)
             for (int s = 0; s < n_stages && ok; ++s) {
                 ok = mbar_wait<RUDDER_SLEEP_MMA>(x_full(sx), phx, abortp, W_X_FULL) &&
                      mbar_wait<RUDDER_SLEEP_MMA>(w_full(sw), phw, abortp, W_W_FULL);
@@ -340,10 +380,30 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ row scales of the tile -> shared
-        if (p.pdl) griddep_wait();                     // so do the row scales
-        for (int i = lane; i < TT; i += 32) rs_smem[i] = (m0 + i < p.M) ? ld_f32_volatile(p.row_scale + m0 + i) : 0.0f;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(rs_full);
+        if (PERSIST) {
+            // one tile ahead of the drain warps, two slots
+            bool ok = true;
+            int it = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += tile_step, ++it) {
+                int m0, n0;
+                tile_origin(tile, m0, n0);
+                const int slot = it & 1;
+                ok = mbar_wait<RUDDER_SLEEP_PROD>(rsp_empty(slot), ((it >> 1) & 1) ^ 1u, abortp, W_RS_FULL);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                for (int i = lane; i < TT; i += 32) rs_smem[slot * TT + i] = (m0 + i < p.M) ? ld_f32_volatile(p.row_scale + m0 + i) : 0.0f;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(rsp_full(slot));
+            }
+        }
+        if (!PERSIST) {
+            int m0, n0;
+            tile_origin(blockIdx.x, m0, n0);
+            if (p.pdl) griddep_wait();                 // so do the row scales
+            for (int i = lane; i < TT; i += 32) rs_smem[i] = (m0 + i < p.M) ? ld_f32_volatile(p.row_scale + m0 + i) : 0.0f;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(rs_full);
+        }
     } else if (warp == 3) {
         // ------------------------------------------------------------------ TMA producer (packed weights)
         // The weights do not depend on the prologue kernel: this stream starts at once.  Channels past N
@@ -354,13 +414,17 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             bool ok = true;
             int slot = 0;
             uint32_t ph = 0;
-            for (int s = 0; s < n_stages; ++s) {
-                ok = mbar_wait<RUDDER_SLEEP_PROD>(raw_empty(slot), ph ^ 1u, abortp, W_RAW_EMPTY);
-                if (!ok) break;
-                mbar_expect_tx(raw_full(slot), p.w_tx);
-                tma_load_2d(smem_base + T::OFF_RAW + slot * RAW_BYTES, p.tm_w, (s0 + s) * (KSTAGE / 2), n0, raw_full(slot));
-                ++issued;
-                if (++slot == SR) { slot = 0; ph ^= 1u; }
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += tile_step) {
+                int m0, n0;
+                tile_origin(tile, m0, n0);
+                for (int s = 0; s < n_stages; ++s) {
+                    ok = mbar_wait<RUDDER_SLEEP_PROD>(raw_empty(slot), ph ^ 1u, abortp, W_RAW_EMPTY);
+                    if (!ok) break;
+                    mbar_expect_tx(raw_full(slot), p.w_tx);
+                    tma_load_2d(smem_base + T::OFF_RAW + slot * RAW_BYTES, p.tm_w, (s0 + s) * (KSTAGE / 2), n0, raw_full(slot));
+                    ++issued;
+                    if (++slot == SR) { slot = 0; ph ^= 1u; }
+                }
             }
             if (!ok) {
                 for (int i = max(0, issued - SR); i < issued; ++i)
@@ -372,22 +436,16 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // 128 channels x 64 packed bytes per stage = 512 16-byte pieces, 4 per thread: piece idx covers
         // channel idx / 4, input channels [32 (idx % 4), 32 (idx % 4) + 32) of the stage.
         const int tid = threadIdx.x - 128;
-        const size_t row_bytes = static_cast<size_t>(p.K / 2);
-        const uint8_t* src[4];
-        bool valid[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int idx = i * UNPACK_THREADS + tid;
-            const int row = idx >> 2, ch = idx & 3;
-            valid[i] = (n0 + row) < p.N;
-            src[i] = p.codes + static_cast<size_t>(valid[i] ? n0 + row : 0) * row_bytes + ch * 16;
-        }
-        // PD stages of packed weights are in flight per thread (registers), so that the L2 / DRAM latency
-        // of the weight stream is covered even when a stage is consumed quickly.
         if (T::RAW) {
             bool ok = true;
             int sw = 0, sr = 0;
             uint32_t phw = 0, phr = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += tile_step) {
+            int m0, n0;
+            tile_origin(tile, m0, n0);
+            bool valid[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) valid[i] = (n0 + ((i * UNPACK_THREADS + tid) >> 2)) < p.N;
             for (int s = 0; s < n_stages && ok; ++s) {
                 ok = mbar_wait<RUDDER_SLEEP_UNPACK>(raw_full(sr), phr, abortp, W_RAW_FULL);
                 if (!ok) break;
@@ -418,7 +476,22 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 if (++sw == SW) { sw = 0; phw ^= 1u; }
                 if (++sr == SR) { sr = 0; phr ^= 1u; }
             }
+            }
         } else {
+        // PD stages of packed weights are in flight per thread (registers), so that the L2 / DRAM latency
+        // of the weight stream is covered even when a stage is consumed quickly.
+        int m0, n0;
+        tile_origin(blockIdx.x, m0, n0);
+        const size_t row_bytes = static_cast<size_t>(p.K / 2);
+        const uint8_t* src[4];
+        bool valid[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int idx = i * UNPACK_THREADS + tid;
+            const int row = idx >> 2, ch = idx & 3;
+            valid[i] = (n0 + row) < p.N;
+            src[i] = p.codes + static_cast<size_t>(valid[i] ? n0 + row : 0) * row_bytes + ch * 16;
+        }
         constexpr int PD = T::PD;
         uint4 pre[PD][4];
         auto load_stage = [&](int s, uint4 (&dst)[4]) {
@@ -474,6 +547,13 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         const int q = warp & 3;                  // TMEM lane quadrant this warp may read
         const int h = (warp - 8) >> 2;           // token half
         const int ch_local = q * 32 + lane;      // channel within the tile = TMEM lane
+        int buf = 0;                             // TMEM buffer of the next group and its phase: carried across tiles
+        uint32_t phb = 0;
+        bool ok = true;
+        int tile_it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += tile_step, ++tile_it) {
+        int m0, n0;
+        tile_origin(tile, m0, n0);
         const int n = n0 + ch_local;
         const bool n_ok = n < p.N;
         float acc[EC];
@@ -484,14 +564,11 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // (Packed two-lane FMAs measured the same: the drain is bound by the FMA pipe and the register
         // file's write port, which the TMEM loads share, not by issue slots.)
         const float sc_mul = F8 ? 16.0f : 1.0f;
-        bool ok = true;
         // Scales are fetched two groups ahead with volatile loads: a plain load would be sunk next to
         // its use and expose the L2 latency once per group.
         const float* sc_ptr = p.scales_t + static_cast<size_t>(g0) * p.N + (n_ok ? n : 0);
         float sc_next = ldg_f32_volatile(sc_ptr);
         float sc_next2 = (n_groups > 1) ? ldg_f32_volatile(sc_ptr + p.N) : 0.0f;
-        int buf = 0;
-        uint32_t phb = 0;
         int g = 0;
         if (NCH == 1 && !DUMP) {
             // Small tiles: a group is one TMEM load per thread, so the fixed cost of a hand-shake (barrier
@@ -592,6 +669,48 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             if (lane == 0) mbar_arrive(acc_empty(buf));  // one arrival per warp: arrivals on one barrier serialise
             if (++buf == T::NBUF) { buf = 0; phb ^= 1u; }
         }
+        if (PERSIST) {
+            // The tile leaves through one slab of 128 tokens x 128 channels, half a tile at a time (the
+            // token half h = 0 first), each half written by one TMA store.  A half is staged once the store
+            // that last used the slab has read it; the wait for the second half's store is left to the next
+            // tile, whose MMAs are running all the while.
+            const float b = (p.bias != nullptr && n_ok) ? __ldg(p.bias + n) : 0.0f;
+            const uint32_t slab = smem_base + T::OFF_OUT;
+            const int rs_slot = tile_it & 1;
+            if (ok) ok = mbar_wait<32>(rsp_full(rs_slot), (tile_it >> 1) & 1, abortp, W_RS_FULL);
+            const float4* rs4 = reinterpret_cast<const float4*>(rs_smem + rs_slot * TT + h * EC);
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass) {
+                if (threadIdx.x == 256) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+                if (h == pass && ok) {
+                    if (ch_local < p.out_pitch) {
+                        uint32_t dst = slab + static_cast<uint32_t>(ch_local) * 2u;
+                        const uint32_t step = static_cast<uint32_t>(p.out_pitch) * 2u;
+#pragma unroll
+                        for (int j = 0; j < EC; j += 4) {
+                            const float4 rs = rs4[j >> 2];                   // broadcast read, zero past M
+                            sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 0], rs.x, b)))); dst += step;
+                            sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 1], rs.y, b)))); dst += step;
+                            sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 2], rs.z, b)))); dst += step;
+                            sts16(dst, __bfloat16_as_ushort(__float2bfloat16_rn(fmaf(acc[j + 3], rs.w, b)))); dst += step;
+                        }
+                    }
+                    fence_proxy_async_smem();                    // generic writes -> visible to the TMA store
+                }
+                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+                if (threadIdx.x == 256) {
+                    const int t0 = m0 + pass * EC;
+                    if (ok && t0 < p.M)
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                     ::"l"(reinterpret_cast<uint64_t>(&tm_y)), "r"(slab), "r"(n0), "r"(t0) : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(rsp_empty(rs_slot));      // this warp has read its row scales
+            continue;
+        }
         // Split K: publish this split's partial sums; the CTA that arrives last at the tile's counter adds
         // the splits in order and goes on to write the tile, the others are done.
         bool writer = true;
@@ -686,6 +805,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         }
+        }   // tile loop (one pass unless PERSIST)
+        if (PERSIST && threadIdx.x == 256) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -700,10 +821,10 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 
 }  // namespace
 
-template <int TT, bool DUMP, bool F8>
+template <int TT, bool DUMP, bool F8, bool PERSIST>
 static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaStream_t st)
 {
-    using T = Tile<TT>;
+    using T = Tile<TT, PERSIST>;
     Params p;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.G;
     p.codes = a.w_codes; p.scales_t = a.w_scales_t;
@@ -722,7 +843,8 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
     p.pdl = plan.pdl ? 1 : 0;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.m_tiles * p.n_tiles, plan.splitk, 1);
+    const int tiles = p.m_tiles * p.n_tiles;
+    cfg.gridDim = dim3(PERSIST ? min(tiles, max(1, a.sm_count)) : tiles, plan.splitk, 1);
     cfg.blockDim = dim3(NUM_THREADS, 1, 1);
     cfg.dynamicSmemBytes = T::DYN_SMEM;
     cfg.stream = st;
@@ -731,16 +853,22 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = plan.pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_kernel<TT, DUMP, F8>, a.tm_x, a.tm_y, p);
+    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_kernel<TT, DUMP, F8, PERSIST>, a.tm_x, a.tm_y, p);
 }
 
 // Tile and split choice.  Large M: 256-token tiles, no split.  M <= 256: the smallest tile that holds
 // the rows, and K split so that about one CTA per SM streams weights, as long as every split keeps at
 // least two stages and the fp32 partials stay small (they must also fit the fixed scratch of
 // rudder_linear_static).
-GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump)
+GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool dump)
 {
     GemmI8Plan plan;
+    // The persistent form pays where the drain warps are idle during the main loop (one scale per output
+    // channel: a single group per tile) and a CTA gets several tiles; measured slower everywhere else.
+    {
+        const long long tiles = static_cast<long long>((M + 255) / 256) * ((N + BN - 1) / BN);
+        plan.persist = !dump && M > 256 && G >= K && G >= RUDDER_PERSIST_MIN_G && tiles >= 3 * 148;
+    }
     plan.token_tile = M > 256 ? 256 : (M > 32 ? 64 : 32);    // up to 256 tokens: small tiles, eight TMEM buffers
     plan.splitk = 1;
     plan.pdl = false;
@@ -760,7 +888,7 @@ GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump)
 
 size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_offset)
 {
-    const GemmI8Plan plan = gemm_i8_plan(M, N, K, dump);
+    const GemmI8Plan plan = gemm_i8_plan(M, N, K, 0, dump);
     const int n_tiles = (N + BN - 1) / BN;
     const int m_tiles = (M + plan.token_tile - 1) / plan.token_tile;
     size_t partial = 0;
@@ -774,24 +902,27 @@ size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_of
 cudaError_t gemm_i8_init()
 {
     cudaError_t e;
-#define RUDDER_I8_ATTR(TT, D)                                                                                                 \
-    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT>::DYN_SMEM); \
-    if (e != cudaSuccess) return e;                                                                                           \
-    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT>::DYN_SMEM);  \
+#define RUDDER_I8_ATTR1(TT, D, F, P)                                                                                                  \
+    e = cudaFuncSetAttribute(gemm_i8_w4_kernel<TT, D, F, P>, cudaFuncAttributeMaxDynamicSharedMemorySize, Tile<TT, P>::DYN_SMEM); \
     if (e != cudaSuccess) return e;
+#define RUDDER_I8_ATTR(TT, D) RUDDER_I8_ATTR1(TT, D, false, false) RUDDER_I8_ATTR1(TT, D, true, false)
     RUDDER_I8_ATTR(32, false) RUDDER_I8_ATTR(64, false) RUDDER_I8_ATTR(256, false)
     RUDDER_I8_ATTR(32, true) RUDDER_I8_ATTR(64, true) RUDDER_I8_ATTR(256, true)
+    RUDDER_I8_ATTR1(256, false, false, true) RUDDER_I8_ATTR1(256, false, true, true)
 #undef RUDDER_I8_ATTR
+#undef RUDDER_I8_ATTR1
     return cudaSuccess;
 }
 
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st)
 {
-    const GemmI8Plan plan = gemm_i8_plan(a.M, a.N, a.K, a.acc != nullptr);
+    const GemmI8Plan plan = gemm_i8_plan(a.M, a.N, a.K, a.G, a.acc != nullptr);
     const bool dump = a.acc != nullptr;
+    if (plan.persist)
+        return a.f8 ? launch_one<256, false, true, true>(a, plan, st) : launch_one<256, false, false, true>(a, plan, st);
 #define RUDDER_I8_LAUNCH(TT)                                                                                     \
-    return a.f8 ? (dump ? launch_one<TT, true, true>(a, plan, st) : launch_one<TT, false, true>(a, plan, st))   \
-                : (dump ? launch_one<TT, true, false>(a, plan, st) : launch_one<TT, false, false>(a, plan, st));
+    return a.f8 ? (dump ? launch_one<TT, true, true, false>(a, plan, st) : launch_one<TT, false, true, false>(a, plan, st))   \
+                : (dump ? launch_one<TT, true, false, false>(a, plan, st) : launch_one<TT, false, false, false>(a, plan, st));
     switch (plan.token_tile) {
         case 32:  RUDDER_I8_LAUNCH(32)
         case 64:  RUDDER_I8_LAUNCH(64)

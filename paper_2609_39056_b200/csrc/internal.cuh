@@ -104,6 +104,7 @@ struct GemmI8Args {
     CUtensorMap tm_y;           // output bf16 [M, N] (row pitch ldy), box {min(128, N) channels, token tile}
     uint16_t* y;                // the same output as a plain pointer (small tiles are stored without TMA)
     int64_t ldy;
+    int sm_count;               // CTAs of the persistent form
     bool f8;                    // E4M3 operands (exact small integers), FP32 accumulators
     const CUtensorMap* tm_w;    // device-resident tensor map over the packed weights (256-token tiles stage them by TMA)
     const uint8_t* w_codes;     // packed INT4 weights
@@ -121,8 +122,9 @@ struct GemmI8Plan {
     int token_tile;             // tokens per CTA tile: sizes the TMA boxes
     int splitk;                 // K splits
     bool pdl;                   // launched with programmatic dependent launch after the prologue kernel
+    bool persist;               // persistent form (256-token tiles): one CTA per SM walks the tiles; output store boxes of 128 tokens
 };
-GemmI8Plan gemm_i8_plan(int M, int N, int K, bool dump);
+GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool dump);
 size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_offset);
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st);
 cudaError_t gemm_i8_init();     // one-time function attributes (dynamic shared memory opt-in)
