@@ -192,7 +192,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
 
     int8_t* codes = static_cast<int8_t*>(workspace);
     float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
-    const GemmI8Plan plan = gemm_i8_plan(M, w->N, w->K, w->G, acc != nullptr);
+    const GemmI8Plan plan = gemm_i8_plan(M, w->N, w->K, w->G, w->f8 != 0, acc != nullptr);
     GemmI8Args g;
     g.partials = nullptr; g.counters = nullptr;
     if (plan.splitk > 1) {
@@ -214,7 +214,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
         return RUDDER_ERR_CUDA;
     if (!make_tmap_2d(&g.tm_y, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, static_cast<uint64_t>(w->N), static_cast<uint64_t>(M),
                       static_cast<uint64_t>(ldy) * 2, static_cast<uint32_t>(w->N < 128 ? w->N : 128),
-                      plan.persist ? static_cast<uint32_t>(M < 128 ? M : 128) : box_tok, CU_TENSOR_MAP_SWIZZLE_NONE))
+                      plan.persist ? 64u : box_tok, CU_TENSOR_MAP_SWIZZLE_NONE))
         return RUDDER_ERR_CUDA;
     g.sm_count = sm_count();
     g.w_codes = w->codes; g.w_scales_t = w->scales_t; g.tm_w = w->tm_codes; g.f8 = w->f8 != 0;

@@ -122,9 +122,9 @@ struct GemmI8Plan {
     int token_tile;             // tokens per CTA tile: sizes the TMA boxes
     int splitk;                 // K splits
     bool pdl;                   // launched with programmatic dependent launch after the prologue kernel
-    bool persist;               // persistent form (256-token tiles): one CTA per SM walks the tiles; output store boxes of 128 tokens
+    bool persist;               // persistent form (256-token tiles): one CTA per SM walks the tiles; output store boxes of 64 tokens
 };
-GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool dump);
+GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool f8, bool dump);
 size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_offset);
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st);
 cudaError_t gemm_i8_init();     // one-time function attributes (dynamic shared memory opt-in)

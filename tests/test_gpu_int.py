@@ -164,16 +164,17 @@ def test_w4a4_extreme_sums_are_exact(rd, G, M):
     _assert_clean(rd)
 
 
-@pytest.mark.parametrize("scheme,mode", [("w4a8", 0), ("w4a8", 1), ("w4a4", 0)])
-def test_per_channel_many_tiles_sampled_rows(rd, scheme, mode):
-    """One scale per output channel (Eq. 10 as printed) over enough tiles (18 x 27) that the GEMM runs in its
-    persistent form: every CTA walks several tiles, ragged last token tile and last channel tile included.
-    The oracle is evaluated on a seeded sample of rows that covers every token tile, first and last rows."""
+@pytest.mark.parametrize("scheme,mode,G", [("w4a8", 0, 384), ("w4a8", 1, 384), ("w4a4", 0, 384), ("w4a8", 0, 128), ("w4a8", 1, 128)])
+def test_many_tiles_persistent_form(rd, scheme, mode, G):
+    """One scale per output channel (Eq. 10 as printed; G = K = 384) and groups of 128, over enough tiles
+    (18 x 27) that the GEMM runs in its persistent form: every CTA walks several tiles, ragged last token
+    tile and last channel tile included.  The oracle is evaluated on a seeded sample of rows that covers
+    every token tile, first and last rows."""
     M, K, N = 4420, 384, 3392
     inp = wl.tiny(seed=4242, M=M, K=K, N=N, T=2)
-    ref_w = oracle.pack_int4(inp.W, inp.d, K)
+    ref_w = oracle.pack_int4(inp.W, inp.d, G)
     clip = static_clip(inp, ref_w["dinv"]) if mode == 1 else None
-    g = GpuLinear(rd, inp, scheme, K, mode, clip)
+    g = GpuLinear(rd, inp, scheme, G, mode, clip)
     Y = rd.rudder_linear(g.w, g.X, g.seg, 1, g.tab, g.bias)
     rng = np.random.default_rng(7)
     rows = np.unique(np.concatenate([[0, 1, 255, 256, 257, M - 2, M - 1], np.arange(0, M, 256) + 3,
@@ -187,7 +188,7 @@ def test_per_channel_many_tiles_sampled_rows(rd, scheme, mode):
     # and its INT32 sums on the sampled rows are the oracle's
     Y2, acc = rd.rudder_linear_dump_acc(g.w, g.X, g.seg, 1, g.tab, g.bias)
     assert torch.equal(Y, Y2)
-    racc = oracle.accumulate_int(out["codes"], ref_w["qw"], K)
+    racc = oracle.accumulate_int(out["codes"], ref_w["qw"], G)
     assert np.array_equal(acc.cpu().numpy()[:, rows, :], racc)
     _assert_clean(rd)
 
