@@ -9,7 +9,7 @@ action) tokens, 10 steps of tables).  The W4A8 block (configuration 2), the W4A4
 (configuration 3) and the small-M sweep (configuration 4) are measured in the same run and reported
 under "also" (rank 0, N = 1).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg2_g128|cfg2_perchannel|cfg2_perchannel_static|cfg3|cfg3_nvfp4|cfg4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg2_g128|cfg2_perchannel|cfg2_perchannel_static|cfg3|cfg3_perchannel|cfg3_nvfp4|cfg4] [--impl reference]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded row sample.
 """
@@ -60,6 +60,10 @@ def workload_config(name: str):
         # paper's sensitivity study (per-output-channel W4, static per-tensor A8)
         suffix = "_g128" if g else ("_per_channel_static" if name.endswith("_static") else "_per_channel")
         return dataclasses.replace(c, name=c.name + suffix, group=g)
+    if name == "cfg3_perchannel":                     # configuration 3 (W4A4-INT) with one scale per output channel
+        import dataclasses
+        c = wl.config(3, "w4a4")
+        return dataclasses.replace(c, name=c.name + "_per_channel", group=0)
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -421,7 +425,7 @@ def run_ours(args):
         del m, ws, tabs, biases, xs, ys, workspace, lins
         torch.cuda.empty_cache()
         also = {}
-        for name in ("cfg2", "cfg2_g128", "cfg2_perchannel", "cfg2_perchannel_static", "cfg3", "cfg3_nvfp4"):
+        for name in ("cfg2", "cfg2_g128", "cfg2_perchannel", "cfg2_perchannel_static", "cfg3", "cfg3_perchannel", "cfg3_nvfp4"):
             if name == args.workload:
                 continue
             c2 = workload_config(name)
