@@ -72,6 +72,9 @@ constexpr int KSTAGE = 128;      // input channels (= bytes of int8 per row) per
 #ifndef RUDDER_PSW
 #define RUDDER_PSW 3             // persistent form: unpacked-weight stages
 #endif
+#ifndef RUDDER_PERSIST_MIN_TILES
+#define RUDDER_PERSIST_MIN_TILES (3 * 148)   // fewest tiles for which the persistent form is used
+#endif
 #ifndef RUDDER_PERSIST_MIN_G
 #define RUDDER_PERSIST_MIN_G 0   // (build-time switch: a huge value turns the persistent form off)
 #endif
@@ -879,7 +882,7 @@ GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool f8, bool dump)
 #else
         const bool shape_ok = G >= K || (G >= 128 && !f8);
 #endif
-        plan.persist = !dump && M > 256 && shape_ok && G >= RUDDER_PERSIST_MIN_G && tiles >= 3 * 148;
+        plan.persist = !dump && M > 256 && shape_ok && G >= RUDDER_PERSIST_MIN_G && tiles >= RUDDER_PERSIST_MIN_TILES;
     }
     plan.token_tile = M > 256 ? 256 : (M > 32 ? 64 : 32);    // up to 256 tokens: small tiles, eight TMEM buffers
     plan.splitk = 1;
