@@ -217,7 +217,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
                       plan.persist ? 64u : box_tok, CU_TENSOR_MAP_SWIZZLE_NONE))
         return RUDDER_ERR_CUDA;
     g.sm_count = sm_count();
-    g.w_codes = w->codes; g.w_scales_t = w->scales_t; g.tm_w = w->tm_codes; g.f8 = w->f8 != 0;
+    g.w_scales_t = w->scales_t; g.tm_w = w->tm_codes; g.f8 = w->f8 != 0;
     g.y = Y; g.ldy = ldy;
     g.M = M; g.N = w->N; g.K = w->K; g.G = w->G;
     g.row_scale = r; g.bias = bias;

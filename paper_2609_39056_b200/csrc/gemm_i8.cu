@@ -20,11 +20,11 @@
 // Warp roles (warpgroup-aligned so that registers can be moved between them):
 //   warp 0        TMA producer: activation codes (int8 [TT tokens][128 B], 128-byte swizzle)
 //   warp 1        allocates TMEM; one lane issues tcgen05.mma kind::i8 (M = 128, N = TT, K = 32)
-//   warp 3        (256-token tiles) TMA producer of the packed INT4 weights: a ring of raw stages
-//                 [128 channels][64 B], several stages ahead of the unpack warps
-//   warps 4-7     take the packed INT4 weights (256-token tiles: from the raw ring; small tiles: from
-//                 global memory / L2 into registers, several stages ahead), expand them to int8 and store
-//                 them in the swizzled K-major layout the tensor core reads.  The nibble goes to the TOP half of the byte (value 16 q): two logic ops
+//   warp 3        TMA producer of the packed INT4 weights: a ring of raw stages [128 channels][64 B],
+//                 several stages ahead of the unpack warps (the weights do not depend on the prologue
+//                 kernel, so this stream starts while that kernel is still running)
+//   warps 4-7     take the packed INT4 weights from the raw ring, expand them to int8 and store them in
+//                 the swizzled K-major layout the tensor core reads.  The nibble goes to the TOP half of the byte (value 16 q): two logic ops
 //                 per 8 weights, no sign extension; the factor 16 is folded into the fp32 scales.
 //   warps 8-15    epilogue: per weight group, drain the INT32 partial sums from TMEM and accumulate
 //                 fp32(C) * Delta_W[j,g] in registers; finally * r_i + b_j -> bf16, transposed through
@@ -36,12 +36,12 @@
 // Shared memory rings (stage = 128 input channels):
 //   X  [SX][TT tokens][128 B]     int8, swizzled by TMA       full: TMA bytes     empty: umma commit
 //   W  [SW][128 channels][128 B]  int8 x16, swizzled by hand  full: 4 warps       empty: umma commit
-//   RAW[SR][128 channels][64 B]   packed INT4, as in memory   full: TMA bytes     empty: 4 warps  (256-token tiles)
+//   RAW[SR][128 channels][64 B]   packed INT4, as in memory   full: TMA bytes     empty: 4 warps
 // 256-token tiles: the output tile [256 tokens][128 channels] bf16 is staged over the X ring once the last
 // MMA is done.
 // Small M (up to 256 tokens: action / proprio-only passes): the token tile shrinks to 32 / 64 and the K
 // dimension is split over blockIdx.y so that about one CTA per SM streams its own slice of the
-// weights, several stages of packed weights in flight per thread.  Each split writes its fp32 partial
+// weights.  Each split writes its fp32 partial
 // tile [token][channel]; the CTA that arrives last at the tile's counter adds the partials in split
 // order (deterministic) and stores its bf16 results straight from registers.  The kernel is launched
 // with programmatic dependent launch: everything that does not read the prologue's output (barrier
@@ -101,13 +101,11 @@ constexpr int RUDDER_SLEEP_EPI = 0;
 template <int TT, bool PERSIST = false> struct Tile {
     static constexpr int SX = PERSIST ? RUDDER_PSX : ((TT == 256) ? 4 : 8);
     static constexpr int SW = PERSIST ? RUDDER_PSW : 4;  // unpacked-weight stages
-    static constexpr int PD = (TT <= 64) ? 4 : 1;    // stages of packed weights a thread keeps in flight
     static constexpr int X_BYTES = TT * KSTAGE;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + SX * X_BYTES;
-    static constexpr bool RAW = (TT == 256);         // packed weights staged by TMA (one more ring) instead of registers
     static constexpr int OFF_RAW = OFF_W + SW * W_BYTES;
-    static constexpr int OFF_OUT = OFF_RAW + (RAW ? SR * RAW_BYTES : 0);
+    static constexpr int OFF_OUT = OFF_RAW + SR * RAW_BYTES;
     static constexpr int OUT_BYTES = 128 * BN * 2;   // persistent form: half a tile of bf16 results
     static constexpr int BYTES = OFF_OUT + (PERSIST ? OUT_BYTES : 0);
     static constexpr int DYN_SMEM = BYTES + 1024;    // slack to align the base to 1024 bytes
@@ -121,7 +119,6 @@ template <int TT, bool PERSIST = false> struct Tile {
 
 struct Params {
     int M, N, K, G;
-    const uint8_t* codes;        // packed INT4 weights [N][K/2], 32-channel interleave (E4M3 path: sign-magnitude words)
     const float* scales_t;       // [K/G][N] fp32 = Delta_W / 16
     const float* row_scale;      // r [M]
     const float* bias;           // [N] or nullptr
@@ -134,15 +131,14 @@ struct Params {
     int m_tiles, n_tiles;        // token tiles, channel tiles (grid.x = m_tiles * n_tiles)
     int splitk;                  // K splits (grid.y)
     int stages_per_split;        // 128-channel stages per split
-    union {                      // (shared storage for the same reason as above: a launch uses one of them)
-        float* partials;         // tiles of 32 / 64 tokens: [splitk][m_tiles * TT][N] fp32 partial sums (splitk > 1)
-        const CUtensorMap* tm_w; // 256-token tiles: tensor map (device memory) over the packed weights, box {64 B, 128 channels}
-    };
+    float* partials;             // tiles of 32 / 64 tokens: [splitk][m_tiles * TT][N] fp32 partial sums (splitk > 1)
+    const CUtensorMap* tm_w;     // tensor map (device memory) over the packed weights, box {64 B, 128 channels}
     int* counters;               // [m_tiles * n_tiles] arrivals per tile, zeroed by the prologue kernel
-    int pdl;                     // launched with programmatic dependent launch
-    uint32_t x_tx;               // bytes one activation TMA box delivers
-    int out_pitch;               // channels per row of the staged output tile (= TMA store box width)
-    uint32_t w_tx;               // bytes one packed-weight TMA box delivers (256-token tiles)
+    // (16-bit fields: the block must stay within the size above)
+    uint16_t pdl;                // launched with programmatic dependent launch
+    uint16_t x_rows;             // token rows one activation TMA box delivers (128 bytes each)
+    uint16_t out_pitch;          // channels per row of the staged output tile (= TMA store box width)
+    uint16_t w_rows;             // channel rows one packed-weight TMA box delivers (64 bytes each)
 };
 static_assert(sizeof(Params) <= 120, "kernel parameters beyond 376 bytes slow the 256-token kernel");
 
@@ -165,12 +161,6 @@ __device__ __forceinline__ void sts16(uint32_t addr, uint16_t v) {
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint4 ldg_nc_16(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
 __device__ __forceinline__ float ldg_f32_volatile(const float* p) {
@@ -278,8 +268,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         for (int i = 0; i < SW; ++i) { mbar_init(w_full(i), UNPACK_THREADS / 32); mbar_init(w_empty(i), 1); }
         for (int i = 0; i < T::NBUF; ++i) { mbar_init(acc_full(i), 1); mbar_init(acc_empty(i), EPI_THREADS / 32); }
         mbar_init(rs_full, 1);
-        if (T::RAW)
-            for (int i = 0; i < SR; ++i) { mbar_init(raw_full(i), 1); mbar_init(raw_empty(i), UNPACK_THREADS / 32); }
+        for (int i = 0; i < SR; ++i) { mbar_init(raw_full(i), 1); mbar_init(raw_empty(i), UNPACK_THREADS / 32); }
         if (PERSIST)
             for (int i = 0; i < 2; ++i) { mbar_init(rsp_full(i), 1); mbar_init(rsp_empty(i), EPI_THREADS / 32); }
         fence_mbar_init();
@@ -315,7 +304,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 for (int s = 0; s < n_stages; ++s) {
                     ok = mbar_wait<RUDDER_SLEEP_PROD>(x_empty(slot), ph ^ 1u, abortp, W_X_EMPTY);
                     if (!ok) break;
-                    mbar_expect_tx(x_full(slot), p.x_tx);
+                    mbar_expect_tx(x_full(slot), static_cast<uint32_t>(p.x_rows) * KSTAGE);
                     tma_load_2d(smem_base + T::OFF_X + slot * T::X_BYTES, &tm_x, (s0 + s) * KSTAGE, m0, x_full(slot));
                     ++issued;
                     if (++slot == T::SX) { slot = 0; ph ^= 1u; }
@@ -411,7 +400,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // ------------------------------------------------------------------ TMA producer (packed weights)
         // The weights do not depend on the prologue kernel: this stream starts at once.  Channels past N
         // are zero-filled by the copy.
-        if (T::RAW && lane == 0) {
+        if (lane == 0) {
             tma_prefetch_desc(p.tm_w);
             int issued = 0;
             bool ok = true;
@@ -423,7 +412,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 for (int s = 0; s < n_stages; ++s) {
                     ok = mbar_wait<RUDDER_SLEEP_PROD>(raw_empty(slot), ph ^ 1u, abortp, W_RAW_EMPTY);
                     if (!ok) break;
-                    mbar_expect_tx(raw_full(slot), p.w_tx);
+                    mbar_expect_tx(raw_full(slot), static_cast<uint32_t>(p.w_rows) * (KSTAGE / 2));
                     tma_load_2d(smem_base + T::OFF_RAW + slot * RAW_BYTES, p.tm_w, (s0 + s) * (KSTAGE / 2), n0, raw_full(slot));
                     ++issued;
                     if (++slot == SR) { slot = 0; ph ^= 1u; }
@@ -439,7 +428,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
         // 128 channels x 64 packed bytes per stage = 512 16-byte pieces, 4 per thread: piece idx covers
         // channel idx / 4, input channels [32 (idx % 4), 32 (idx % 4) + 32) of the stage.
         const int tid = threadIdx.x - 128;
-        if (T::RAW) {
+        {
             bool ok = true;
             int sw = 0, sr = 0;
             uint32_t phw = 0, phr = 0;
@@ -480,65 +469,6 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
                 if (++sr == SR) { sr = 0; phr ^= 1u; }
             }
             }
-        } else {
-        // PD stages of packed weights are in flight per thread (registers), so that the L2 / DRAM latency
-        // of the weight stream is covered even when a stage is consumed quickly.
-        int m0, n0;
-        tile_origin(blockIdx.x, m0, n0);
-        const size_t row_bytes = static_cast<size_t>(p.K / 2);
-        const uint8_t* src[4];
-        bool valid[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int idx = i * UNPACK_THREADS + tid;
-            const int row = idx >> 2, ch = idx & 3;
-            valid[i] = (n0 + row) < p.N;
-            src[i] = p.codes + static_cast<size_t>(valid[i] ? n0 + row : 0) * row_bytes + ch * 16;
-        }
-        constexpr int PD = T::PD;
-        uint4 pre[PD][4];
-        auto load_stage = [&](int s, uint4 (&dst)[4]) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                dst[i] = valid[i] ? ldg_nc_16(src[i] + static_cast<size_t>(s0 + s) * (KSTAGE / 2)) : make_uint4(0, 0, 0, 0);
-        };
-#pragma unroll
-        for (int j = 0; j < PD; ++j)
-            if (j < n_stages) load_stage(j, pre[j]);
-        bool ok = true;
-        int sw = 0;
-        uint32_t phw = 0;
-        for (int sb = 0; sb < n_stages && ok; sb += PD) {
-#pragma unroll
-            for (int j = 0; j < PD; ++j) {
-                const int s = sb + j;
-                if (s < n_stages && ok) {
-                    uint4 cur[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) cur[i] = pre[j][i];
-                    if (s + PD < n_stages) load_stage(s + PD, pre[j]);
-                    ok = mbar_wait<RUDDER_SLEEP_UNPACK>(w_empty(sw), phw ^ 1u, abortp, W_W_EMPTY);
-                    if (ok) {
-                        const uint32_t dst = smem_base + T::OFF_W + sw * W_BYTES;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int idx = i * UNPACK_THREADS + tid;
-                            const int row = idx >> 2, ch = idx & 3;
-                            const uint4 pk = cur[i];
-                            uint4 lo, hi;
-                            unpack32<F8>(pk, lo, hi);
-                            const uint32_t drow = dst + (row >> 3) * 1024 + (row & 7) * 128;
-                            sts128(drow + (((2 * ch) ^ (row & 7)) << 4), lo);
-                            sts128(drow + (((2 * ch + 1) ^ (row & 7)) << 4), hi);
-                        }
-                        fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(w_full(sw));      // one arrival per warp: arrivals on one barrier serialise
-                        if (++sw == SW) { sw = 0; phw ^= 1u; }
-                    }
-                }
-            }
-        }
         }
     }
     } else {
@@ -836,18 +766,19 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
     using T = Tile<TT, PERSIST>;
     Params p;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.G;
-    p.codes = a.w_codes; p.scales_t = a.w_scales_t;
+    p.scales_t = a.w_scales_t;
     p.row_scale = a.row_scale; p.bias = a.bias;
     if (DUMP) { p.aux.dump.acc = a.acc; p.aux.dump.row0 = a.row0; p.aux.dump.rows = a.rows; p.aux.dump.col0 = a.col0; p.aux.dump.cols = a.cols; }
     else      { p.aux.out.y = a.y; p.aux.out.ldy = a.ldy; }
-    p.x_tx = static_cast<uint32_t>(min(TT, a.M)) * KSTAGE;
-    p.out_pitch = min(BN, a.N);
-    p.w_tx = static_cast<uint32_t>(min(BN, a.N)) * (KSTAGE / 2);
+    p.x_rows = static_cast<uint16_t>(min(TT, a.M));
+    p.out_pitch = static_cast<uint16_t>(min(BN, a.N));
+    p.w_rows = static_cast<uint16_t>(min(BN, a.N));
     p.m_tiles = (a.M + TT - 1) / TT;
     p.n_tiles = (a.N + BN - 1) / BN;
     p.splitk = plan.splitk;
     p.stages_per_split = a.K / KSTAGE / plan.splitk;
-    if (T::RAW) p.tm_w = a.tm_w; else p.partials = a.partials;
+    p.tm_w = a.tm_w;
+    p.partials = a.partials;
     p.counters = a.counters;
     p.pdl = plan.pdl ? 1 : 0;
 

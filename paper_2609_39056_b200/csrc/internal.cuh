@@ -107,7 +107,6 @@ struct GemmI8Args {
     int sm_count;               // CTAs of the persistent form
     bool f8;                    // E4M3 operands (exact small integers), FP32 accumulators
     const CUtensorMap* tm_w;    // device-resident tensor map over the packed weights (256-token tiles stage them by TMA)
-    const uint8_t* w_codes;     // packed INT4 weights
     const float* w_scales_t;    // [K/G][N]
     int M, N, K, G;
     const float* row_scale;     // r [M]
