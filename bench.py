@@ -74,7 +74,9 @@ def algorithmic_bytes_linear(M, K, N, G, scheme):
         act = M * K // 2 + M * K // 16 + 4 * M
         w = N * K // 2 + N * K // 16 + 4
     else:
-        act = M * K + 4 * M           # one code per byte in the workspace (both integer schemes)
+        # b_a bits per code: the method's 8 or 4.  (The W4A4-INT path keeps one code per BYTE in its
+        # workspace, twice this: the difference shows up as traffic above the algorithmic bytes.)
+        act = M * K * (8 if scheme == "w4a8" else 4) // 8 + 4 * M
         w = N * K // 2 + 2 * N * K // (G or K)       # G = 0: one scale per output channel
     return 2 * M * K + 2 * act + w + 2 * M * N + 4 * N
 
@@ -238,7 +240,7 @@ def roofline_of(cfg, m, pk):
     if cfg.scheme == "nvfp4":
         pro_bytes = sum(2 * M * K + M * K // 2 + M * K // 16 + 4 * M for _, K, N in cfg.linears)
     else:
-        pro_bytes = sum(2 * M * K + M * K + 4 * M for _, K, N in cfg.linears)
+        pro_bytes = sum(2 * M * K + M * K * (8 if cfg.scheme == "w4a8" else 4) // 8 + 4 * M for _, K, N in cfg.linears)
     traffic = NCU_TRAFFIC_BYTES.get(cfg.name)
     return {"kernel": "gemm_nvfp4_pair_kernel" if cfg.scheme == "nvfp4" else "gemm_i8_w4_kernel", "launches_per_step": 4,
             "bound": "tensor", "achieved": achieved, "peak": tensor_peak,
