@@ -28,6 +28,8 @@ def _layers(rd):
         GpuLinear(rd, wl.tiny(seed=903, M=200, K=512, N=256, T=2), "nvfp4", 16),
         GpuLinear(rd, wl.tiny(seed=904, M=300, K=1024, N=384, T=2), "w4a8", 128),    # 256-token tiles, TMA store
         GpuLinear(rd, wl.tiny(seed=905, M=1030, K=512, N=256, T=2), "nvfp4", 16),    # CTA-pair kernel
+        GpuLinear(rd, wl.tiny(seed=906, M=4420, K=256, N=3392, T=2), "w4a8", 256),   # 486 tiles, one scale per channel: persistent form
+        GpuLinear(rd, wl.tiny(seed=907, M=4420, K=256, N=3392, T=2), "w4a8", 128),   # persistent form with two groups per tile
     ]
 
 
@@ -46,7 +48,7 @@ def test_chain_shares_workspace(rd):
                                g.inp.bias)
     check_output(bf16_to_np(alone[0]), out["y64"], rel=REL_TOL, abs_=ABS_TOL)
 
-    order = [0, 1, 2, 3, 4, 0, 0, 2, 4, 4, 1, 3, 3, 1, 0, 2, 2, 4, 0]
+    order = [0, 1, 2, 3, 4, 0, 0, 2, 4, 4, 1, 3, 3, 1, 0, 2, 2, 4, 0, 5, 0, 6, 5, 5, 3, 6, 1]
     outs = [torch.full_like(alone[i], float("nan")) for i in order]
     for i, y in zip(order, outs):
         g = layers[i]
