@@ -322,6 +322,30 @@ def small_m_sweep(rd, torch, dev, pk, schemes=("w4a8", "w4a4"), sizes=(2048, 409
     return out
 
 
+def calibrator_timing(rd, torch, dev):
+    """Toy calibrator (Eq. 9) on the QKV layer of configuration 2, one layer-step: wall time of the whole
+    search (every candidate is one static-mode rudder_linear plus the error reduction)."""
+    from paper_2609_39056_b200 import calibrate as gc
+    cfg = wl.config(2)
+    l = cfg.draw()[0]
+    W = torch.from_numpy(l.W).to(dev)
+    d = torch.from_numpy(l.d).to(dev)
+    w = rd.rudder_pack_weights(W, d, rd.SCHEMES[cfg.scheme], l.K)           # one scale per output channel
+    X = torch.from_numpy(l.X_bf16.view(np.int16)).to(dev).view(torch.bfloat16)
+    seg = rd.Segments(l.seg_offsets, l.seg_stream)
+    v = (X.float() * rd.rudder_weight_export(w)["dinv"][None, :]).abs().flatten()
+    cs = [float(torch.kthvalue(v, max(1, int(round(q * v.numel())))).values) for q in (0.99, 0.999, 0.9999, 1.0)]
+    steps = [2 ** -0.5, 2 ** -0.25, 2 ** 0.25, 2 ** 0.5]
+    gc.calibrate_step(w, X, seg, 3, cs[:1], steps[:1], sweeps=1)            # warm-up
+    torch.cuda.synchronize()
+    t0 = time.time()
+    r = gc.calibrate_step(w, X, seg, 3, cs, steps)
+    torch.cuda.synchronize()
+    dt = time.time() - t0
+    return {"layer": "cfg2 qkv 4416x2048x6144, per-channel W4A8, static range", "ms": dt * 1e3, "evaluations": r["evaluations"],
+            "gamma": [float(g) for g in r["gamma"]], "clip": r["clip"], "objective": r["objective"]}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -440,6 +464,7 @@ def run_ours(args):
             del m2
             torch.cuda.empty_cache()
         also["cfg4_small_m_sweep"] = small_m_sweep(rd, torch, dev, pk)
+        also["toy_calibrator"] = calibrator_timing(rd, torch, dev)
 
     if rank == 0:
         line = {
