@@ -150,12 +150,20 @@ typedef struct {
     const rudder_weight* w[4];
     const rudder_scale_table* tab[4];
     const float* bias[4];        /* each [N_l] or NULL */
-    const uint16_t* x[4];        /* replay inputs, bf16 [M, ldx[l]] */
+    const uint16_t* x[4];        /* replay inputs, bf16 [M, ldx[l]]; x[1..3] may be NULL: chained (see below) */
     int64_t ldx[4];
     uint16_t* y[4];              /* outputs, bf16 [M, ldy[l]] */
     int64_t ldy[4];
 } rudder_block_args;
 
+/* Chained layers.  x[l] == NULL for l = 1, 2 or 3 makes that layer read the previous layer's output
+ * through the minimal BF16 glue, so that the block runs end to end on the device from x[0] alone:
+ *   O    (l = 1): the V third of the QKV output, y[0][:, 2 K_1 .. 3 K_1) -- a stand-in for attention, which
+ *                 stays outside this library; requires N_0 == 3 K_1;
+ *   up   (l = 2): the O output as it is (no norm / residual); requires N_1 == K_2;
+ *   down (l = 3): rudder_gelu of the up output, staged at the end of the workspace; requires N_2 == K_3.
+ * A shape that does not chain returns RUDDER_ERR_SHAPE.  rudder_block_workspace_bytes accounts for the
+ * staged GELU output (M x K_3 bf16) when x[3] is NULL.  rudder_block_host takes no NULL inputs. */
 size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M);
 rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
                            void* workspace, size_t workspace_bytes, void* stream);
@@ -198,6 +206,16 @@ rudder_status rudder_linear_dump_acc(const rudder_weight* w, const uint16_t* X, 
                                      const float* bias, uint16_t* Y, int64_t ldy,
                                      void* workspace, size_t workspace_bytes, void* stream,
                                      int row0, int rows, int col0, int cols, int32_t* acc);
+
+/* BF16 GELU, elementwise, Y = bf16(gelu(X)): the glue of a chained block (the paper keeps GELU in BF16,
+ * Appendix "Quantization"; which GELU is not stated).  Reading: the tanh form
+ *   gelu(x) = x/2 (1 + tanh(0.7978845608 (x + 0.044715 x^3)))
+ * with tanh u replaced by its [7/6] Pade approximant
+ *   u (135135 + 17325 u^2 + 378 u^4 + u^6) / (135135 + 62370 u^2 + 3150 u^4 + 28 u^6)   for |u| < 5, +-1 beyond,
+ * evaluated in fp32 by Horner's rule from the highest power, every add, multiply and the one divide
+ * rounded to nearest on its own (no fused multiply-add): the result is defined bit for bit.
+ * X, Y bf16 [M, ld]; N % 8 == 0; 16-byte aligned pointers, leading dimensions multiples of 8. */
+rudder_status rudder_gelu(const uint16_t* X, int64_t ldx, int M, int N, uint16_t* Y, int64_t ldy, void* stream);
 
 /* Reads and clears the device status word (SYNCHRONISES the device).  *last (HOST) receives
  * RUDDER_OK or RUDDER_ERR_TIMEOUT; *where (HOST, may be NULL) a code naming the wait that gave up. */

@@ -27,6 +27,7 @@ EXPORTED = [
     "rudder_linear_static_max_workspace_bytes", "rudder_linear_static",
     "rudder_block_profile", "rudder_block_host_staging_bytes", "rudder_block_host",
     "rudder_quantize_activations", "rudder_linear_dump_acc", "rudder_device_status", "rudder_status_string",
+    "rudder_gelu",
 ]
 
 
@@ -93,6 +94,7 @@ def lib() -> ctypes.CDLL:
                                              ctypes.POINTER(_ScaleTable), vp, vp, i64, vp, sz, vp,
                                              i32, i32, i32, i32, vp]
         L.rudder_device_status.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.rudder_gelu.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         _lib = L
     return _lib
 
@@ -270,11 +272,21 @@ class BlockArgs:
             c.w[l] = weights[l].handle
             c.tab[l] = ctypes.pointer(tabs[l].c)
             c.bias[l] = biases[l].data_ptr() if biases[l] is not None else None
-            c.x[l] = xs[l].data_ptr()
-            c.ldx[l] = xs[l].stride(0)
+            c.x[l] = xs[l].data_ptr() if xs[l] is not None else None        # None (l >= 1): chained to the previous output
+            c.ldx[l] = xs[l].stride(0) if xs[l] is not None else 0
             c.y[l] = ys[l].data_ptr()
             c.ldy[l] = ys[l].stride(0)
         self.c = c
+
+
+def rudder_gelu(X: torch.Tensor, Y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Y = bf16(gelu(X)), elementwise, in the bit-defined form the chained block uses."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    M, N = X.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    _check(lib().rudder_gelu(_ptr(X), X.stride(0), int(M), int(N), _ptr(Y), Y.stride(0), _stream(stream)), "rudder_gelu")
+    return Y
 
 
 def rudder_block_workspace_bytes(args: BlockArgs, M: int) -> int:

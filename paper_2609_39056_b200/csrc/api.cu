@@ -403,6 +403,8 @@ size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M)
         if (!args->w[l]) return 0;
         total += workspace_bytes_for(args->w[l], M);
     }
+    if (args->x[3] == nullptr)       // chained: GELU(up output) is staged here as the down projection's input
+        total += align_up(static_cast<size_t>(M) * args->w[3]->K * 2, 256);
     return total;
 }
 
@@ -411,23 +413,49 @@ static rudder_status block_impl(const rudder_block_args* args, int M, const rudd
 {
     if (!args) return RUDDER_ERR_ARG;
     for (int l = 0; l < 4; ++l)
-        if (!args->w[l] || !args->tab[l] || !args->x[l] || !args->y[l]) return RUDDER_ERR_ARG;
+        if (!args->w[l] || !args->tab[l] || (!args->x[l] && l == 0) || !args->y[l]) return RUDDER_ERR_ARG;
     const size_t need = rudder_block_workspace_bytes(args, M);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < need || need == 0) return RUDDER_ERR_WORKSPACE;
+    // Chained layers (x[l] == NULL, l >= 1) take the previous output through the minimal glue: the V third
+    // of the QKV output stands in for attention, the O output feeds the up projection as it is, GELU of the
+    // up output (staged at the end of the workspace) feeds the down projection.
+    const uint16_t* x_eff[4];
+    int64_t ldx_eff[4];
+    size_t lin_bytes = 0;
+    for (int l = 0; l < 4; ++l) lin_bytes += workspace_bytes_for(args->w[l], M);
+    uint16_t* gelu_buf = reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + lin_bytes);
+    for (int l = 0; l < 4; ++l) {
+        x_eff[l] = args->x[l];
+        ldx_eff[l] = args->ldx[l];
+        if (args->x[l] != nullptr) continue;
+        const int K = args->w[l]->K, Np = args->w[l - 1]->N;
+        if (l == 1) {
+            if (Np != 3 * K) return RUDDER_ERR_SHAPE;
+            x_eff[l] = args->y[0] + 2 * static_cast<size_t>(K);
+            ldx_eff[l] = args->ldy[0];
+        } else {
+            if (Np != K) return RUDDER_ERR_SHAPE;
+            x_eff[l] = (l == 3) ? gelu_buf : args->y[l - 1];
+            ldx_eff[l] = (l == 3) ? K : args->ldy[l - 1];
+        }
+    }
     // validate everything before the first launch
     for (int l = 0; l < 4; ++l) {
         SegParams sp;
         rudder_status s = check_table_and_segments(seg, step, args->tab[l], M, &sp);
         if (s != RUDDER_OK) return s;
         const rudder_weight* w = args->w[l];
-        if (!aligned(args->x[l], 16) || !aligned(args->y[l], 16) || args->ldx[l] % 8 != 0 || args->ldy[l] % 8 != 0 ||
-            args->ldx[l] < w->K || args->ldy[l] < w->N)
+        if (!aligned(x_eff[l], 16) || !aligned(args->y[l], 16) || ldx_eff[l] % 8 != 0 || args->ldy[l] % 8 != 0 ||
+            ldx_eff[l] < w->K || args->ldy[l] < w->N)
             return RUDDER_ERR_ALIGN;
     }
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     for (int l = 0; l < 4; ++l) {
         const size_t bytes = workspace_bytes_for(args->w[l], M);
-        rudder_status s = linear_impl(args->w[l], args->x[l], args->ldx[l], M, seg, step, args->tab[l], args->bias[l],
+        if (l == 3 && args->x[3] == nullptr &&
+            launch_gelu(args->y[2], args->ldy[2], gelu_buf, args->w[3]->K, M, args->w[3]->K, sm_count(), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return RUDDER_ERR_CUDA;
+        rudder_status s = linear_impl(args->w[l], x_eff[l], ldx_eff[l], M, seg, step, args->tab[l], args->bias[l],
                                       args->y[l], args->ldy[l], ws, bytes, static_cast<cudaStream_t>(stream), nullptr, 0, 0,
                                       0, 0, ev ? ev + 2 * l : nullptr);
         if (s != RUDDER_OK) return s;
@@ -590,6 +618,16 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
     if (launch_actq_int(a, qmax_of(w->scheme), false, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     return RUDDER_OK;
+}
+
+rudder_status rudder_gelu(const uint16_t* X, int64_t ldx, int M, int N, uint16_t* Y, int64_t ldy, void* stream)
+{
+    if (!X || !Y) return RUDDER_ERR_ARG;
+    if (M < 1 || N < 8 || N % 8 != 0) return RUDDER_ERR_SHAPE;
+    if (!aligned(X, 16) || !aligned(Y, 16) || ldx % 8 != 0 || ldy % 8 != 0 || ldx < N || ldy < N) return RUDDER_ERR_ALIGN;
+    rudder_status s = ensure_init();
+    if (s != RUDDER_OK) return s;
+    return launch_gelu(X, ldx, Y, ldy, M, N, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? RUDDER_OK : RUDDER_ERR_CUDA;
 }
 
 rudder_status rudder_device_status(int* last, int* where)

@@ -1,0 +1,80 @@
+// BF16 glue between the quantized linears of a chained DiT block (the paper keeps GELU in BF16,
+// outside the quantized path: Appendix "Quantization").  Only what a chain of rudder_linear calls
+// needs to run back to back on the device: an elementwise GELU.
+//
+// GELU is taken in its tanh form, g(x) = x/2 (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))), with tanh
+// replaced by its [7/6] Pade approximant
+//     tanh u ~ u (135135 + 17325 u^2 + 378 u^4 + u^6) / (135135 + 62370 u^2 + 3150 u^4 + 28 u^6)
+// for |u| < 5 and by +-1 beyond (error below 2e-4 of the tanh form, under the bf16 step of the
+// result).  Every operation is a single correctly rounded fp32 add, multiply or divide in the order
+// written below -- no fused multiply-add, no approximate instruction -- so that the result is
+// defined bit for bit and a plain CPU program can repeat it.
+#include "internal.cuh"
+
+#include <cuda_bf16.h>
+
+namespace rudder {
+
+namespace {
+
+__device__ __forceinline__ float gelu_f32(float x) {
+    const float x2 = __fmul_rn(x, x);
+    const float x3 = __fmul_rn(x2, x);
+    const float inner = __fadd_rn(x, __fmul_rn(0.044715f, x3));
+    const float u = __fmul_rn(0.7978845608028654f, inner);
+    float t;
+    if (!(fabsf(u) < 5.0f)) {
+        t = (u < 0.0f) ? -1.0f : 1.0f;              // also +-infinity; NaN propagates through the product below
+        if (u != u) t = u;
+    } else {
+        const float u2 = __fmul_rn(u, u);
+        float n = __fadd_rn(u2, 378.0f);
+        n = __fadd_rn(__fmul_rn(n, u2), 17325.0f);
+        n = __fadd_rn(__fmul_rn(n, u2), 135135.0f);
+        n = __fmul_rn(n, u);
+        float d = __fadd_rn(__fmul_rn(28.0f, u2), 3150.0f);
+        d = __fadd_rn(__fmul_rn(d, u2), 62370.0f);
+        d = __fadd_rn(__fmul_rn(d, u2), 135135.0f);
+        t = __fdiv_rn(n, d);
+    }
+    return __fmul_rn(__fmul_rn(0.5f, x), __fadd_rn(1.0f, t));
+}
+
+__device__ __forceinline__ uint32_t gelu_pair(uint32_t w) {
+    const float lo = gelu_f32(__uint_as_float(w << 16));
+    const float hi = gelu_f32(__uint_as_float(w & 0xFFFF0000u));
+    return static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(lo))) |
+           (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(hi))) << 16);
+}
+
+// One 16-byte chunk (8 values) per thread step; rows of N values (N % 8 == 0), leading dimensions in elements.
+__global__ void __launch_bounds__(256) gelu_bf16_kernel(const uint16_t* __restrict__ X, int64_t ldx, uint16_t* __restrict__ Y, int64_t ldy,
+                                                        int M, int N)
+{
+    const int chunks = N >> 3;
+    const long long total = static_cast<long long>(M) * chunks;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int row = static_cast<int>(i / chunks);
+        const int c = static_cast<int>(i - static_cast<long long>(row) * chunks);
+        const uint4 v = *reinterpret_cast<const uint4*>(X + static_cast<size_t>(row) * ldx + 8 * c);
+        uint4 o;
+        o.x = gelu_pair(v.x); o.y = gelu_pair(v.y); o.z = gelu_pair(v.z); o.w = gelu_pair(v.w);
+        *reinterpret_cast<uint4*>(Y + static_cast<size_t>(row) * ldy + 8 * c) = o;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_gelu(const uint16_t* X, int64_t ldx, uint16_t* Y, int64_t ldy, int M, int N, int sm_count, cudaStream_t st)
+{
+    const long long total = static_cast<long long>(M) * (N >> 3);
+    long long blocks = (total + 255) / 256;
+    const long long cap = static_cast<long long>(sm_count > 0 ? sm_count : 148) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    gelu_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(X, ldx, Y, ldy, M, N);
+    return cudaGetLastError();
+}
+
+}  // namespace rudder

@@ -68,6 +68,7 @@ cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G
                              cudaStream_t st);
 cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, bool signmag, cudaStream_t st);
 
+cudaError_t launch_gelu(const uint16_t* X, int64_t ldx, uint16_t* Y, int64_t ldy, int M, int N, int sm_count, cudaStream_t st);
 cudaError_t actq_init();
 // e4m3: the codes (integers in [-7, 7]) are written as E4M3 bytes for the FP8 tensor path instead of int8
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, bool e4m3, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);

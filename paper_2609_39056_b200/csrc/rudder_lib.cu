@@ -9,5 +9,6 @@
 #include "gemm_i8.cu"
 #include "gemm_fp4.cu"
 #include "gemm_fp4_pair.cu"
+#include "glue.cu"
 #include "api.cu"
 #include "static_ws.cu"

@@ -1,0 +1,82 @@
+"""BF16 glue on the GPU: the GELU kernel against the oracle on every bf16 bit pattern, and the chained
+block (x[1..3] = NULL) against the same four linears and the glue run one by one."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from helpers import GpuLinear, bf16_to_np, check_output, oracle_pack, to_dev_bf16
+from oracle import glue
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rd():
+    import paper_2609_39056_b200 as rd
+    rd.lib()
+    return rd
+
+
+def test_gelu_every_bf16_pattern(rd):
+    bits = np.arange(65536, dtype=np.uint16).reshape(512, 128)
+    X = to_dev_bf16(bits)
+    Y = rd.rudder_gelu(X)
+    got = bf16_to_np(Y)
+    want = glue.gelu_bf16(bits)
+    x = glue.bf16_to_f32(bits)
+    finite = np.isfinite(x)
+    assert np.array_equal(got[finite], want[finite])
+    # infinities and NaN: same class of result (NaN payloads are not compared)
+    g, w = glue.bf16_to_f32(got[~finite]), glue.bf16_to_f32(want[~finite])
+    assert np.array_equal(np.isnan(g), np.isnan(w)) and np.array_equal(g[~np.isnan(g)], w[~np.isnan(w)])
+
+
+def test_gelu_strided_and_errors(rd):
+    X = torch.randn((37, 256), device="cuda").to(torch.bfloat16)
+    Y = torch.full((37, 384), 7.0, dtype=torch.bfloat16, device="cuda")
+    rd.rudder_gelu(X[:, 64:192], Y[:, 128:256])
+    want = glue.gelu_bf16(bf16_to_np(X[:, 64:192].contiguous()))
+    assert np.array_equal(bf16_to_np(Y[:, 128:256].contiguous()), want)
+    assert torch.all(Y[:, :128] == 7.0) and torch.all(Y[:, 256:] == 7.0)
+    with pytest.raises(rd.RudderError):
+        rd.rudder_gelu(X[:, :100])              # N not a multiple of 8
+
+
+@pytest.mark.parametrize("scheme,G", [("w4a8", 64), ("nvfp4", 16)])
+def test_chained_block(rd, scheme, G):
+    H, F, M = 256, 1024, 70
+    shapes = [(H, 3 * H), (H, H), (H, F), (F, H)]
+    layers = [GpuLinear(rd, wl.tiny(seed=700 + i, M=M, K=K, N=N, T=2), scheme, G) for i, (K, N) in enumerate(shapes)]
+    seg, step = layers[0].seg, 1
+    # one by one, with the same glue
+    y0 = rd.rudder_linear(layers[0].w, layers[0].X, seg, step, layers[0].tab, layers[0].bias)
+    y1 = rd.rudder_linear(layers[1].w, y0[:, 2 * H:3 * H], seg, step, layers[1].tab, layers[1].bias)
+    y2 = rd.rudder_linear(layers[2].w, y1, seg, step, layers[2].tab, layers[2].bias)
+    a2 = rd.rudder_gelu(y2)
+    y3 = rd.rudder_linear(layers[3].w, a2, seg, step, layers[3].tab, layers[3].bias)
+    # chained
+    ys = [torch.full_like(y, float("nan")) for y in (y0, y1, y2, y3)]
+    bargs = rd.BlockArgs([l.w for l in layers], [l.tab for l in layers], [l.bias for l in layers],
+                         [layers[0].X, None, None, None], ys)
+    ws = torch.empty(rd.rudder_block_workspace_bytes(bargs, M) + 256, dtype=torch.uint8, device="cuda")
+    rd.rudder_block(bargs, M, seg, step, ws)
+    torch.cuda.synchronize()
+    for l, (a, b) in enumerate(zip(ys, (y0, y1, y2, y3))):
+        assert torch.equal(a, b), f"layer {l}"
+    # each layer against the oracle, fed the GPU's own input of that layer
+    ins = [bf16_to_np(layers[0].X), bf16_to_np(y0[:, 2 * H:3 * H].contiguous()), bf16_to_np(y1), glue.gelu_bf16(bf16_to_np(y2))]
+    assert np.array_equal(ins[3], bf16_to_np(a2))
+    for l, g in enumerate(layers):
+        ref_w = oracle_pack(g.inp, scheme, G)
+        out = oracle.rudder_linear(ins[l], ref_w, g.inp.gamma, None, step, 0, layers[0].inp.seg_offsets, layers[0].inp.seg_stream,
+                                   scheme, g.inp.bias)
+        check_output(bf16_to_np(ys[l]), out["y64"], **({"rel": 2e-2} if scheme == "nvfp4" else {}))
+    # a shape that does not chain is refused before anything is launched
+    bad = rd.BlockArgs([layers[0].w, layers[2].w, layers[2].w, layers[3].w], [l.tab for l in layers], [None] * 4,
+                       [layers[0].X, None, None, None], ys)
+    with pytest.raises(rd.RudderError):
+        rd.rudder_block(bad, M, seg, step, ws)
+    last, where = rd.rudder_device_status()
+    assert last == 0, (last, where)
