@@ -258,6 +258,103 @@ def test_p4_nvfp4_error_bound():
     assert sb.max() <= 0x7E and e.max() <= 15
 
 
+# ------------------------------------------------------------------------------------------ P4 (NVFP4 recipe)
+# The paper only names NVFP4, so the recipe is a reading; what the reading *means* is still fixed by
+# mathematics: a block's scale is the block maximum divided by the largest E2M1 magnitude (6), rounded
+# to UE4M3 (3 mantissa bits: relative error at most 2^-4), so the block's largest element lands in
+# 6 x [1/(1+2^-4), 1/(1-2^-4)] = [5.65, 6.4] and must take the end code +-6; every other element is the
+# nearest E2M1 value of (value / outer scale) / block scale; the outer scale maps the tensor's (row's)
+# largest magnitude to 6 x 448 = 2688.  A wrong divisor, a dropped outer scale or a wrong table fails here.
+_E2M1 = np.array([0, .5, 1, 1.5, 2, 3, 4, 6])
+
+
+def _nvfp4_check(V, e, sb, outer_scale, what):
+    """V fp64 [R, K] (the values that were quantised), e codes [R, K], sb UE4M3 bytes [R, K/16],
+    outer_scale fp32 [R] (the fp32 scale of each row: tensor scale or row scale)."""
+    R, K = V.shape
+    sbd = np.array([oracle.ue4m3_decode(b) for b in range(127)])[sb]                 # decoded block scales
+    amax_b = np.abs(V).reshape(R, K // 16, 16).max(-1)
+    # (d) outer scale x 2688 = largest magnitude of the row / tensor, to fp32 rounding
+    live = outer_scale > 0
+    # (a) normal, unsaturated block scale -> the block's absmax element carries code 7 (+-6)
+    normal = (sb >= 8) & (sb <= 0x7E)
+    mag = (e & 7).reshape(R, K // 16, 16)
+    arg = np.abs(V).reshape(R, K // 16, 16).argmax(-1)
+    top_code = np.take_along_axis(mag, arg[..., None], -1)[..., 0]
+    assert normal.sum() > 0.5 * normal.size, what
+    assert np.all(top_code[normal] == 7), f"{what}: a block maximum is not encoded as +-6"
+    # (b) the dequantised block maximum is the block's true maximum within the UE4M3 rounding (2^-4)
+    deq_top = 6.0 * sbd * outer_scale[:, None].astype(np.float64)
+    unsat = normal & (sb < 0x7E)
+    assert np.all(np.abs(deq_top - amax_b)[unsat] <= amax_b[unsat] * (2.0 ** -4) * (1 + 1e-5)), what
+    # (c) every code is the nearest E2M1 value of (V / outer) / block scale (near-ties left out: the oracle
+    #     forms the quotient in fp32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        u = V / outer_scale[:, None].astype(np.float64) / np.repeat(sbd, 16, 1)
+    ok = np.isfinite(u)
+    au = np.minimum(np.abs(u), 6.0)
+    nearest = np.abs(au[..., None] - _E2M1).argmin(-1)
+    mids = np.array([.25, .75, 1.25, 1.75, 2.5, 3.5, 5.0])
+    near_tie = (np.abs(au[..., None] - mids) <= 1e-5 * np.maximum(au[..., None], 1.0)).any(-1)
+    sel = ok & ~near_tie
+    assert sel.mean() > 0.9, what
+    assert np.array_equal((e & 7)[sel], nearest[sel]), f"{what}: a code is not the nearest E2M1 value"
+    sign_ok = ((e >> 3) == (V < 0))[sel & ((e & 7) != 0)]
+    assert sign_ok.all(), what
+    # zero block scale -> zero codes
+    assert not (e.reshape(R, K // 16, 16)[sb == 0]).any(), what
+    return live
+
+
+def test_p4_nvfp4_weight_recipe():
+    inp = wl.tiny(seed=31, M=4, K=512, N=96)
+    pw = oracle.pack_nvfp4(inp.W, inp.d)
+    V32 = inp.W * inp.d[None, :]                                   # fp32 product, as the fold defines it
+    V = V32.astype(np.float64)
+    ts = np.float32(pw["tensor_scale"])
+    np.testing.assert_allclose(float(ts) * 2688.0, np.abs(V32).max(), rtol=2e-7)     # (d)
+    _nvfp4_check(V, pw["e2m1"], pw["sb"], np.full(inp.N, ts, np.float32), "weights")
+    # the block that holds the tensor's largest magnitude saturates the scale format: 448, code 0x7E
+    j, k = np.unravel_index(np.abs(V32).argmax(), V32.shape)
+    assert pw["sb"][j, k // 16] == 0x7E and (pw["e2m1"][j, k] & 7) == 7
+    # canonical nibble packing: low nibble = even k
+    assert np.array_equal(pw["packed"], (pw["e2m1"][:, 0::2] | (pw["e2m1"][:, 1::2] << 4)).astype(np.uint8))
+
+
+@pytest.mark.parametrize("mode", [PT, ST])
+def test_p4_nvfp4_activation_recipe(mode):
+    inp = wl.tiny(seed=32, M=24, K=512, N=64, T=2)
+    dinv = (np.float32(1) / inp.d).astype(np.float32)
+    clip = _static_clip(inp, dinv) if mode == ST else None
+    step = 1
+    e, sb, r = oracle.quantize_nvfp4(inp.X_bf16, dinv, inp.gamma, clip, step, mode, inp.seg_offsets, inp.seg_stream)
+    row_stream = np.repeat(inp.seg_stream, np.diff(inp.seg_offsets))
+    g = inp.gamma[step, row_stream]
+    v32 = (_f32(inp.X_bf16) * dinv[None, :]) * g[:, None]          # gamma X D^-1 in fp32, two rounded products
+    a = np.full(inp.M, clip[step], np.float32) if mode == ST else np.abs(v32).max(1)
+    s_row = (r.astype(np.float64) * g.astype(np.float64)).astype(np.float32)         # r_i = s_i / gamma
+    np.testing.assert_allclose(s_row.astype(np.float64) * 2688.0, a, rtol=3e-7)      # (d)
+    if mode == ST:
+        # values beyond the threshold saturate: block scale 448 where the block maximum exceeds c, codes +-6
+        v = v32.astype(np.float64)
+        over = np.abs(v) > float(clip[step]) * (1 + 1e-6)
+        assert over.any()
+        assert np.all((e & 7)[over] == 7)
+        assert np.all(sb[np.abs(v).reshape(inp.M, -1, 16).max(-1) > float(clip[step]) * (1 + 1e-6)] == 0x7E)
+        keep = np.abs(v).reshape(inp.M, -1, 16).max(-1) <= float(clip[step])
+        # check the recipe on the blocks that do not clip
+        vv = np.where(np.repeat(keep, 16, 1), v, 0.0)
+        ee = np.where(np.repeat(keep, 16, 1), e, 0)
+        ss = np.where(keep, sb, 0)
+        _nvfp4_check(vv, ee.astype(np.uint8), ss.astype(np.uint8), s_row, "activations (static)")
+    else:
+        _nvfp4_check(v32.astype(np.float64), e, sb, s_row, "activations (per token)")
+        # the row's largest element: block scale 448, code +-6 -- it dequantises to a_i exactly
+        top = np.abs(v32).argmax(1)
+        assert np.all(sb[np.arange(inp.M), top // 16] == 0x7E)
+        assert np.all((e[np.arange(inp.M), top] & 7) == 7)
+
+
 # ------------------------------------------------------------------------------------------ P5
 @pytest.mark.parametrize("scheme", ["w4a8", "w4a4", "nvfp4"])
 @pytest.mark.parametrize("mode", [PT, ST])
