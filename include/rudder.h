@@ -22,6 +22,11 @@
  *     status word that rudder_device_status reads.
  *   - bf16 / fp16 values are passed as their 16-bit patterns (uint16_t).
  *   - Non-finite inputs are undefined behaviour (not checked).
+ *   - A rudder_weight belongs to the device that was current when it was packed or imported.  Every call
+ *     that takes one must be made with that device current and with buffers of that device; a call made
+ *     with another device current returns RUDDER_ERR_ARG before anything is launched.
+ *   - Host threads may call concurrently on different streams as long as they share no workspace;
+ *     per-device state that is created on first use is guarded inside the library.
  *
  * Shapes: X is [M, K] row-major with leading dimension ldx (elements), W is [N, K] row-major (K
  * contiguous: the transpose of the paper's W in Y = X W), Y is [M, N] with leading dimension ldy.
@@ -105,6 +110,15 @@ rudder_status rudder_weight_info(const rudder_weight* w, int* N, int* K, int* gr
  *   dinv   fp32 [K];  tensor_scale fp32 [1] (NVFP4; 1.0 otherwise).  Any output may be NULL. */
 rudder_status rudder_weight_export(const rudder_weight* w, uint8_t* codes, void* scales, float* dinv,
                                    float* tensor_scale, void* stream);
+
+/* The inverse of rudder_weight_export: builds a packed weight from its canonical view ("stored as packed
+ * integers with corresponding quantization scales", Section 4.2, last paragraph), e.g. from a checkpoint
+ * written earlier.  Same layouts as above, all DEVICE pointers; tensor_scale is required for NVFP4 and
+ * ignored otherwise; group as in rudder_pack_weights.  The handle behaves exactly like the one
+ * rudder_pack_weights returned for the exported weight (same bits out of every kernel).  Allocates and
+ * SYNCHRONISES the stream, like rudder_pack_weights. */
+rudder_status rudder_weight_import(const uint8_t* codes, const void* scales, const float* dinv, const float* tensor_scale,
+                                   int N, int K, rudder_scheme scheme, int group, void* stream, rudder_weight** out);
 
 /* ---------------------------------------------------------------------------------------------
  * rudder_linear -- one quantized linear layer for one denoising step (Section 4.4; Eq. 8; Eq. 10):
@@ -220,6 +234,12 @@ rudder_status rudder_gelu(const uint16_t* X, int64_t ldx, int M, int N, uint16_t
 /* Reads and clears the device status word (SYNCHRONISES the device).  *last (HOST) receives
  * RUDDER_OK or RUDDER_ERR_TIMEOUT; *where (HOST, may be NULL) a code naming the wait that gave up. */
 rudder_status rudder_device_status(int* last, int* where);
+
+/* Self-test of the bounded-wait path (no counterpart in the paper): launches ONE warp that waits, for at
+ * most limit_cycles SM clocks (1e3 .. 1e8), on a barrier that nothing signals -- no copy, no tensor memory,
+ * nothing in flight -- gives up, records RUDDER_ERR_TIMEOUT with the wait code 901 in the device status word
+ * and returns normally.  The context stays usable; rudder_device_status then reports and clears the word. */
+rudder_status rudder_selftest_wait_timeout(long long limit_cycles, void* stream);
 
 const char* rudder_status_string(rudder_status s);
 

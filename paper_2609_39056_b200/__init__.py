@@ -22,12 +22,12 @@ RANGE_PER_TOKEN, RANGE_STATIC = 0, 1
 SCHEMES = {"w4a8": W4A8_INT, "w4a4": W4A4_INT, "nvfp4": W4A4_NVFP4}
 
 EXPORTED = [
-    "rudder_pack_weights", "rudder_weight_free", "rudder_weight_info", "rudder_weight_export",
+    "rudder_pack_weights", "rudder_weight_free", "rudder_weight_info", "rudder_weight_export", "rudder_weight_import",
     "rudder_linear_workspace_bytes", "rudder_linear", "rudder_block_workspace_bytes", "rudder_block",
     "rudder_linear_static_max_workspace_bytes", "rudder_linear_static",
     "rudder_block_profile", "rudder_block_host_staging_bytes", "rudder_block_host",
     "rudder_quantize_activations", "rudder_linear_dump_acc", "rudder_device_status", "rudder_status_string",
-    "rudder_gelu",
+    "rudder_gelu", "rudder_selftest_wait_timeout",
 ]
 
 
@@ -72,6 +72,7 @@ def lib() -> ctypes.CDLL:
         L.rudder_weight_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
                                          ctypes.POINTER(i32), ctypes.POINTER(sz)]
         L.rudder_weight_export.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.rudder_weight_import.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
         L.rudder_linear_workspace_bytes.restype = sz
         L.rudder_linear_workspace_bytes.argtypes = [vp, i32]
         L.rudder_linear.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32, ctypes.POINTER(_ScaleTable),
@@ -95,6 +96,7 @@ def lib() -> ctypes.CDLL:
                                              i32, i32, i32, i32, vp]
         L.rudder_device_status.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32)]
         L.rudder_gelu.argtypes = [vp, i64, i32, i32, vp, i64, vp]
+        L.rudder_selftest_wait_timeout.argtypes = [ctypes.c_longlong, vp]
         _lib = L
     return _lib
 
@@ -184,12 +186,30 @@ def rudder_weight_export(w: Weight, stream=None):
     return dict(codes=codes, scales=scales, dinv=dinv, tensor_scale=ts)
 
 
+def rudder_weight_import(ex: dict, N: int, K: int, scheme: int, group: int, stream=None) -> Weight:
+    """Packed weight from its canonical view (the dict rudder_weight_export returns)."""
+    out = ctypes.c_void_p()
+    _check(lib().rudder_weight_import(_ptr(ex["codes"]), _ptr(ex["scales"]), _ptr(ex["dinv"]), _ptr(ex.get("tensor_scale")),
+                                      int(N), int(K), int(scheme), int(group), _stream(stream), ctypes.byref(out)),
+           "rudder_weight_import")
+    n, k, g, s, b = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_size_t()
+    _check(lib().rudder_weight_info(out, ctypes.byref(n), ctypes.byref(k), ctypes.byref(g), ctypes.byref(s),
+                                    ctypes.byref(b)), "rudder_weight_info")
+    return Weight(out, n.value, k.value, g.value, s.value, b.value)
+
+
 def rudder_linear_workspace_bytes(w: Weight, M: int) -> int:
     return int(lib().rudder_linear_workspace_bytes(w.handle, int(M)))
 
 
-def _workspace(nbytes, device):
-    return torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+def _workspace(nbytes, device, stream=None):
+    """Scratch the binding allocates for the caller.  It is dropped when the call returns, while the kernels
+    may still be running: torch's caching allocator only hands a freed block to later work of the stream it
+    was allocated on, so the block is allocated under the stream the kernels are launched on."""
+    if stream is None:
+        return torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+    with torch.cuda.stream(stream):
+        return torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
 
 
 def _aligned(ws: torch.Tensor):
@@ -204,7 +224,7 @@ def rudder_linear(w: Weight, X: torch.Tensor, seg: Segments, step: int, tab: Sca
     if Y is None:
         Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=X.device)
     if workspace is None:
-        workspace = _workspace(rudder_linear_workspace_bytes(w, M), X.device)
+        workspace = _workspace(rudder_linear_workspace_bytes(w, M), X.device, stream)
     wp, wb = _aligned(workspace)
     _check(lib().rudder_linear(w.handle, _ptr(X), X.stride(0), M, ctypes.byref(seg.c), int(step), ctypes.byref(tab.c),
                                _ptr(bias), _ptr(Y), Y.stride(0), wp, wb, _stream(stream)), "rudder_linear")
@@ -237,7 +257,7 @@ def rudder_linear_dump_acc(w: Weight, X, seg, step, tab, bias=None, row0=0, rows
     cols = w.N - col0 if cols is None else cols
     Y = torch.empty((M, w.N), dtype=torch.bfloat16, device=X.device)
     acc = torch.full((w.K // w.group, rows, cols), -(2 ** 31), dtype=torch.int32, device=X.device)
-    workspace = _workspace(rudder_linear_workspace_bytes(w, M), X.device)
+    workspace = _workspace(rudder_linear_workspace_bytes(w, M), X.device, stream)
     wp, wb = _aligned(workspace)
     _check(lib().rudder_linear_dump_acc(w.handle, _ptr(X), X.stride(0), M, ctypes.byref(seg.c), int(step),
                                         ctypes.byref(tab.c), _ptr(bias), _ptr(Y), Y.stride(0), wp, wb, _stream(stream),
@@ -326,3 +346,8 @@ def rudder_device_status():
     last, where = ctypes.c_int(), ctypes.c_int()
     _check(lib().rudder_device_status(ctypes.byref(last), ctypes.byref(where)), "rudder_device_status")
     return last.value, where.value
+
+
+def rudder_selftest_wait_timeout(limit_cycles: int = 1_000_000, stream=None):
+    """One warp waits `limit_cycles` SM clocks on a barrier nobody signals, gives up and records the time-out."""
+    _check(lib().rudder_selftest_wait_timeout(int(limit_cycles), _stream(stream)), "rudder_selftest_wait_timeout")

@@ -10,11 +10,35 @@
 #include "internal.cuh"
 #include "fp4.cuh"
 
-#ifndef RUDDER_ROW_NCH
-#define RUDDER_ROW_NCH 2            // blocks of 16 channels per thread of the row kernels
-#endif
+#include <cuda_fp16.h>
+
+constexpr int kRowNch = 2;          // blocks of 16 channels per thread of the row kernels
 
 namespace rudder {
+
+// ---- self-test of the bounded-wait path -------------------------------------------------------------
+// One warp waits, with a short cycle limit, on a barrier that nobody signals (no copy, no tensor memory,
+// nothing in flight), gives up, records the time-out in the device status word and returns.
+constexpr int W_SELFTEST = 901;
+__global__ void wait_timeout_selftest_kernel(long long limit_cycles)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    bool ok = mbar_wait<32>(smem_u32(&bar), 0, &abort_word, W_SELFTEST, limit_cycles);
+    ok = __syncthreads_and(ok) != 0;          // the whole CTA leaves together
+    (void)ok;
+}
+cudaError_t launch_wait_timeout_selftest(long long limit_cycles, cudaStream_t st)
+{
+    wait_timeout_selftest_kernel<<<1, 32, 0, st>>>(limit_cycles);
+    return cudaGetLastError();
+}
 
 __device__ __forceinline__ uint4 ld_nc_16(const uint4* p) {
     uint4 v;
@@ -298,12 +322,14 @@ __device__ __forceinline__ void bulk_row_load(uint32_t dst, const void* src, uin
 // Maximum over the CTA of a non-negative float.  `red` holds three slots that rotate from row to row:
 // slot (i + 1) % 3 is cleared while row i is reduced; it was last read before the barrier of row i - 1,
 // which thread 0 has already passed, and is next written after the barrier of row i.
-__device__ __forceinline__ float cta_max_nonneg(float m, uint32_t* red, int& slot) {
+// `ok` goes through the same barrier (AND over the CTA), so that every thread learns whether any thread
+// gave up its wait for the row and all of them leave the row loop together.
+__device__ __forceinline__ float cta_max_nonneg(float m, uint32_t* red, int& slot, bool& ok) {
     const uint32_t wm = __reduce_max_sync(0xffffffffu, __float_as_uint(m));
     const int nxt = (slot == 2) ? 0 : slot + 1;
     if ((threadIdx.x & 31) == 0) atomicMax(red + slot, wm);
     if (threadIdx.x == 0) red[nxt] = 0u;
-    __syncthreads();
+    ok = __syncthreads_and(ok) != 0;
     const float r = __uint_as_float(*reinterpret_cast<volatile uint32_t*>(red + slot));
     slot = nxt;
     return r;
@@ -467,7 +493,9 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
             continue;
         }
         const int slot = j & (kRowSlots - 1);
-        if (!mbar_wait<20>(bar0 + 8u * slot, (j / kRowSlots) & 1, &abort_word, W_ROW_FULL)) break;
+        // A thread whose wait gave up still walks to the row's barrier, where the verdict becomes common to
+        // the CTA (what it computes from the unfinished row meanwhile is discarded).
+        bool ok = mbar_wait<20>(bar0 + 8u * slot, (j / kRowSlots) & 1, &abort_word, W_ROW_FULL);
         const float g = g_slot[slot];
         const uint32_t src = ring_addr + slot * row_bytes;
 
@@ -484,8 +512,15 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
             m = fmaxf(m, mb[i]);
         }
         float range;
-        if (per_token) range = __fmul_rn(cta_max_nonneg(m, red, slot3), g);
-        else { __syncthreads(); range = clip; }
+        if (per_token) range = __fmul_rn(cta_max_nonneg(m, red, slot3, ok), g);
+        else { ok = __syncthreads_and(ok) != 0; range = clip; }
+        if (!ok) {
+            // let the copies already in flight land before the CTA's shared memory goes away (bounded)
+            if (t == 0)
+                for (int jj = j; jj < n_live && jj < j + kRowSlots; ++jj)
+                    for (uint32_t it = 0; it < (1u << 16) && !mbar_try_wait(bar0 + 8u * (jj & (kRowSlots - 1)), (jj / kRowSlots) & 1); ++it) {}
+            break;
+        }
         // every thread has consumed the staged row: refill its slot
         if (t == 0 && j + kRowSlots < n_live) issue(j + kRowSlots);
         const float inv = (range != 0.0f) ? __fdiv_rn(range_max, range) : 0.0f;
@@ -550,7 +585,7 @@ static cudaError_t launch_early(void (*kernel)(KArgs...), int grid, int block, s
 // Blocks of 16 channels per thread and threads per CTA for a row of n blocks.
 static bool row_launch_shape(int n, int& threads, int& nch) {
     if (n > 1024) return false;
-    nch = n > 512 ? 4 : RUDDER_ROW_NCH;             // long rows: fewer, fatter threads keep two CTAs per SM
+    nch = n > 512 ? 4 : kRowNch;             // long rows: fewer, fatter threads keep two CTAs per SM
     while (nch > 1 && n < 32 * nch) nch >>= 1;      // short rows: keep a full warp busy
     threads = ((n + nch - 1) / nch + 31) / 32 * 32;
     return true;
@@ -591,6 +626,29 @@ static bool launch_row(const ActqArgs& a, const RowOut& o, int rows, cudaStream_
     else if (nch == 2) *err = launch_early(actq_row_kernel<FP4, 2>, row_grid(actq_row_kernel<FP4, 2>, rows, threads, smem), threads, smem, st, a, o);
     else               *err = launch_early(actq_row_kernel<FP4, 4>, row_grid(actq_row_kernel<FP4, 4>, rows, threads, smem), threads, smem, st, a, o);
     return true;
+}
+
+// Parity hook: E4M3 bytes (the form the E4M3 tensor path reads) -> the int8 codes they stand for, in place.
+__global__ void e4m3_to_int8_kernel(uint32_t* __restrict__ codes, size_t n_words)
+{
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n_words; i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+        const uint32_t w = codes[i];
+        uint32_t h01, h23;
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h01) : "h"(static_cast<uint16_t>(w & 0xFFFFu)));
+        asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h23) : "h"(static_cast<uint16_t>(w >> 16)));
+        const __half2 a = *reinterpret_cast<const __half2*>(&h01), b = *reinterpret_cast<const __half2*>(&h23);
+        const int q0 = __half2int_rn(__low2half(a)), q1 = __half2int_rn(__high2half(a));
+        const int q2 = __half2int_rn(__low2half(b)), q3 = __half2int_rn(__high2half(b));
+        codes[i] = (q0 & 0xFF) | ((q1 & 0xFF) << 8) | ((q2 & 0xFF) << 16) | (static_cast<uint32_t>(q3 & 0xFF) << 24);
+    }
+}
+
+cudaError_t launch_e4m3_to_int8(int8_t* codes, size_t n_bytes, cudaStream_t st)
+{
+    const size_t n_words = n_bytes / 4;
+    const int blocks = static_cast<int>(n_words / 256 + 1 < 2048 ? n_words / 256 + 1 : 2048);
+    e4m3_to_int8_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<uint32_t*>(codes), n_words);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st)

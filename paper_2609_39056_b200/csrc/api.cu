@@ -4,7 +4,25 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 using namespace rudder;
+
+namespace rudder {
+int device_sm_count()
+{
+    static std::atomic<int> cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+}  // namespace rudder
 
 namespace {
 
@@ -61,33 +79,33 @@ bool make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t k64, uint64_t atom
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Per-device state created on first use (function attributes, SM count, copy streams, the address of the
+// static workspace): guarded by one mutex, so that host threads may make their first calls concurrently.
+std::mutex g_state_mutex;
 bool g_gemm_ready[64] = {false};
 
-int g_sm_count[64] = {0};
 
-int sm_count()
-{
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64) return 148;
-    if (g_sm_count[dev] == 0) {
-        int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
-        g_sm_count[dev] = n;
-    }
-    return g_sm_count[dev];
-}
+int sm_count() { return rudder::device_sm_count(); }
 
 rudder_status ensure_init()
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (dev < 0 || dev >= 64) return RUDDER_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_state_mutex);
     if (!g_gemm_ready[dev]) {
         if (gemm_i8_init() != cudaSuccess || gemm_fp4_init() != cudaSuccess || actq_init() != cudaSuccess) return RUDDER_ERR_CUDA;
         g_gemm_ready[dev] = true;
     }
     return RUDDER_OK;
+}
+
+// A packed weight lives on the device that was current when it was packed; every call that launches on it
+// must be made with that device current (its tensor maps and pointers mean nothing elsewhere).
+bool on_weights_device(const rudder_weight* w)
+{
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == w->device;
 }
 
 rudder_status check_table_and_segments(const rudder_segments* seg, int step, const rudder_scale_table* tab, int M,
@@ -135,6 +153,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
                           int col0, int cols, cudaEvent_t* ev = nullptr /* ev[1] recorded after the prologue, ev[2] after the GEMM */)
 {
     if (!w || !X || !Y) return RUDDER_ERR_ARG;
+    if (!on_weights_device(w)) return RUDDER_ERR_ARG;
     if (M < 1) return RUDDER_ERR_SHAPE;
     SegParams sp;
     rudder_status s = check_table_and_segments(seg, step, tab, M, &sp);
@@ -246,78 +265,133 @@ const char* rudder_status_string(rudder_status s)
     return "unknown status";
 }
 
+// Shape / scheme checks shared by pack and import; normalises `group` (16 for NVFP4).
+static rudder_status check_weight_shape(int N, int K, rudder_scheme scheme, int* group)
+{
+    if (N < 64 || N % 64 != 0 || K < 128 || K % 128 != 0) return RUDDER_ERR_SHAPE;
+    if (scheme != RUDDER_W4A8_INT && scheme != RUDDER_W4A4_INT && scheme != RUDDER_W4A4_NVFP4) return RUDDER_ERR_UNSUPPORTED;
+    if (scheme == RUDDER_W4A4_NVFP4) {
+        if (K % 256 != 0) return RUDDER_ERR_SHAPE;        // the block-scaled GEMM moves 256 input channels per stage
+        *group = 16;
+    } else if (!(*group == 64 || *group == 128 || *group == K)) {
+        return RUDDER_ERR_SHAPE;
+    }
+    return RUDDER_OK;
+}
+
+// Allocates the handle and its device arrays (nothing is filled in).  nullptr if an allocation failed.
+static rudder_weight* alloc_weight(int N, int K, rudder_scheme scheme, int group)
+{
+    rudder_weight* w = static_cast<rudder_weight*>(calloc(1, sizeof(rudder_weight)));
+    if (!w) return nullptr;
+    w->N = N; w->K = K; w->G = group; w->scheme = scheme;
+    cudaGetDevice(&w->device);
+    const size_t n_groups = static_cast<size_t>(K / group);
+    const size_t code_bytes = static_cast<size_t>(N) * (K / 2);
+    bool ok = cudaMalloc(&w->codes, code_bytes) == cudaSuccess &&
+              cudaMalloc(&w->dinv, static_cast<size_t>(K) * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&w->tensor_scale, sizeof(float)) == cudaSuccess;
+    if (scheme == RUDDER_W4A4_NVFP4) {
+        const size_t sf_bytes = static_cast<size_t>((N + 127) / 128) * (K / 64) * 512;
+        ok = ok && cudaMalloc(&w->scales_c, n_groups * N) == cudaSuccess && cudaMalloc(&w->sf_tiled, sf_bytes) == cudaSuccess;
+        w->bytes = code_bytes + n_groups * N + sf_bytes + static_cast<size_t>(K) * sizeof(float) + sizeof(float);
+    } else {
+        // W4A4 with group scales: |C^(g)| <= 128 * 49, so E4M3 operands and FP32 accumulators hold the
+        // integers exactly and the per-group drain needs no integer-to-float conversion.
+        w->f8 = (scheme == RUDDER_W4A4_INT && group <= 128) ? 1 : 0;
+        ok = ok && cudaMalloc(&w->scales_t, n_groups * N * sizeof(float)) == cudaSuccess &&
+             cudaMalloc(&w->scales_c, n_groups * N * sizeof(uint16_t)) == cudaSuccess &&
+             cudaMalloc(&w->tm_codes, sizeof(CUtensorMap)) == cudaSuccess;
+        w->bytes = code_bytes + n_groups * N * (sizeof(float) + sizeof(uint16_t)) + static_cast<size_t>(K) * sizeof(float) + sizeof(float);
+    }
+    if (!ok) {
+        rudder_weight_free(w);
+        return nullptr;
+    }
+    return w;
+}
+
+// Integer schemes: the tensor map over the packed codes, kept in device memory so that the GEMM takes it by pointer.
+static bool finish_int4(rudder_weight* w)
+{
+    CUtensorMap tm;
+    return make_tmap_2d(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w->codes, static_cast<uint64_t>(w->K / 2), static_cast<uint64_t>(w->N),
+                        static_cast<uint64_t>(w->K / 2), 64, static_cast<uint32_t>(w->N < 128 ? w->N : 128), CU_TENSOR_MAP_SWIZZLE_NONE) &&
+           cudaMemcpy(w->tm_codes, &tm, sizeof(CUtensorMap), cudaMemcpyHostToDevice) == cudaSuccess;
+}
+
 rudder_status rudder_pack_weights(const float* W, const float* d, int N, int K, rudder_scheme scheme, int group,
                                   void* stream, rudder_weight** out)
 {
     if (out) *out = nullptr;
     if (!W || !out) return RUDDER_ERR_ARG;
-    if (N < 64 || N % 64 != 0 || K < 128 || K % 128 != 0) return RUDDER_ERR_SHAPE;
-    if (scheme != RUDDER_W4A8_INT && scheme != RUDDER_W4A4_INT && scheme != RUDDER_W4A4_NVFP4) return RUDDER_ERR_UNSUPPORTED;
-    if (scheme == RUDDER_W4A4_NVFP4) {
-        if (K % 256 != 0) return RUDDER_ERR_SHAPE;        // the block-scaled GEMM moves 256 input channels per stage
-        group = 16;
-    } else if (!(group == 64 || group == 128 || group == K)) {
-        return RUDDER_ERR_SHAPE;
-    }
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rudder_status s = ensure_init();
+    rudder_status s = check_weight_shape(N, K, scheme, &group);
     if (s != RUDDER_OK) return s;
-
-    rudder_weight* w = static_cast<rudder_weight*>(calloc(1, sizeof(rudder_weight)));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = ensure_init();
+    if (s != RUDDER_OK) return s;
+    rudder_weight* w = alloc_weight(N, K, scheme, group);
     if (!w) return RUDDER_ERR_CUDA;
-    w->N = N; w->K = K; w->G = group; w->scheme = scheme;
-    cudaGetDevice(&w->device);
-    const size_t n_groups = static_cast<size_t>(K / group);
-    const size_t code_bytes = static_cast<size_t>(N) * (K / 2);
+    bool ok;
     if (scheme == RUDDER_W4A4_NVFP4) {
         const size_t sf_bytes = static_cast<size_t>((N + 127) / 128) * (K / 64) * 512;
         unsigned int* amax_bits = nullptr;
-        bool ok4 = cudaMalloc(&w->codes, code_bytes) == cudaSuccess &&
-                   cudaMalloc(&w->scales_c, n_groups * N) == cudaSuccess &&
-                   cudaMalloc(&w->sf_tiled, sf_bytes) == cudaSuccess &&
-                   cudaMalloc(&w->dinv, static_cast<size_t>(K) * sizeof(float)) == cudaSuccess &&
-                   cudaMalloc(&w->tensor_scale, sizeof(float)) == cudaSuccess &&
-                   cudaMalloc(&amax_bits, sizeof(unsigned int)) == cudaSuccess;
-        w->bytes = code_bytes + n_groups * N + sf_bytes + static_cast<size_t>(K) * sizeof(float) + sizeof(float);
-        if (ok4)
-            ok4 = launch_pack_nvfp4(W, d, N, K, w->codes, static_cast<uint8_t*>(w->scales_c), w->sf_tiled, sf_bytes, w->dinv,
-                                    w->tensor_scale, amax_bits, st) == cudaSuccess &&
-                  cudaStreamSynchronize(st) == cudaSuccess;
+        ok = cudaMalloc(&amax_bits, sizeof(unsigned int)) == cudaSuccess &&
+             launch_pack_nvfp4(W, d, N, K, w->codes, static_cast<uint8_t*>(w->scales_c), w->sf_tiled, sf_bytes, w->dinv,
+                               w->tensor_scale, amax_bits, st) == cudaSuccess &&
+             cudaStreamSynchronize(st) == cudaSuccess;
         if (amax_bits) cudaFree(amax_bits);
-        if (!ok4) {
-            rudder_weight_free(w);
-            return RUDDER_ERR_CUDA;
-        }
-        *out = w;
-        return RUDDER_OK;
-    }
-    // W4A4 with group scales: |C^(g)| <= 128 * 49, so E4M3 operands and FP32 accumulators hold the
-    // integers exactly and the per-group drain needs no integer-to-float conversion.
-#ifndef RUDDER_NO_F8
-    w->f8 = (scheme == RUDDER_W4A4_INT && group <= 128) ? 1 : 0;
-#endif
-    int8_t* tmp = nullptr;
-    bool ok = cudaMalloc(&w->codes, code_bytes) == cudaSuccess &&
-              cudaMalloc(&w->scales_t, n_groups * N * sizeof(float)) == cudaSuccess &&
-              cudaMalloc(&w->scales_c, n_groups * N * sizeof(uint16_t)) == cudaSuccess &&
-              cudaMalloc(&w->dinv, static_cast<size_t>(K) * sizeof(float)) == cudaSuccess &&
-              cudaMalloc(&w->tensor_scale, sizeof(float)) == cudaSuccess &&
-              cudaMalloc(&tmp, static_cast<size_t>(N) * K) == cudaSuccess;
-    w->bytes = code_bytes + n_groups * N * (sizeof(float) + sizeof(uint16_t)) + static_cast<size_t>(K) * sizeof(float) + sizeof(float);
-    if (ok) {
+    } else {
+        int8_t* tmp = nullptr;
         const float one = 1.0f;
-        ok = cudaMemcpyAsync(w->tensor_scale, &one, sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess &&
+        ok = cudaMalloc(&tmp, static_cast<size_t>(N) * K) == cudaSuccess &&
+             cudaMemcpyAsync(w->tensor_scale, &one, sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess &&
              launch_pack_int4(W, d, N, K, group, w->codes, w->scales_t, static_cast<uint16_t*>(w->scales_c), w->dinv, tmp, w->f8 != 0, st) == cudaSuccess &&
              cudaStreamSynchronize(st) == cudaSuccess;
+        if (tmp) cudaFree(tmp);
+        ok = ok && finish_int4(w);
     }
-    if (tmp) cudaFree(tmp);
-    if (ok) {
-        // tensor map over the packed codes, kept in device memory so that the GEMM takes it by pointer
-        CUtensorMap tm;
-        ok = make_tmap_2d(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w->codes, static_cast<uint64_t>(K / 2), static_cast<uint64_t>(N),
-                          static_cast<uint64_t>(K / 2), 64, static_cast<uint32_t>(N < 128 ? N : 128), CU_TENSOR_MAP_SWIZZLE_NONE) &&
-             cudaMalloc(&w->tm_codes, sizeof(CUtensorMap)) == cudaSuccess &&
-             cudaMemcpy(w->tm_codes, &tm, sizeof(CUtensorMap), cudaMemcpyHostToDevice) == cudaSuccess;
+    if (!ok) {
+        rudder_weight_free(w);
+        return RUDDER_ERR_CUDA;
+    }
+    *out = w;
+    return RUDDER_OK;
+}
+
+rudder_status rudder_weight_import(const uint8_t* codes, const void* scales, const float* dinv, const float* tensor_scale,
+                                   int N, int K, rudder_scheme scheme, int group, void* stream, rudder_weight** out)
+{
+    if (out) *out = nullptr;
+    if (!codes || !scales || !dinv || !out) return RUDDER_ERR_ARG;
+    if (scheme == RUDDER_W4A4_NVFP4 && !tensor_scale) return RUDDER_ERR_ARG;
+    rudder_status s = check_weight_shape(N, K, scheme, &group);
+    if (s != RUDDER_OK) return s;
+    if (!aligned(codes, 4) || !aligned(scales, 2)) return RUDDER_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = ensure_init();
+    if (s != RUDDER_OK) return s;
+    rudder_weight* w = alloc_weight(N, K, scheme, group);
+    if (!w) return RUDDER_ERR_CUDA;
+    const size_t n_groups = static_cast<size_t>(K / group);
+    bool ok = cudaMemcpyAsync(w->dinv, dinv, static_cast<size_t>(K) * sizeof(float), cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+    if (scheme == RUDDER_W4A4_NVFP4) {
+        const size_t sf_bytes = static_cast<size_t>((N + 127) / 128) * (K / 64) * 512;
+        ok = ok && cudaMemcpyAsync(w->codes, codes, static_cast<size_t>(N) * (K / 2), cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+             cudaMemcpyAsync(w->scales_c, scales, n_groups * N, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+             cudaMemcpyAsync(w->tensor_scale, tensor_scale, sizeof(float), cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+             launch_import_nvfp4_scales(static_cast<const uint8_t*>(scales), N, K, w->sf_tiled, sf_bytes, st) == cudaSuccess &&
+             cudaStreamSynchronize(st) == cudaSuccess;
+    } else {
+        int8_t* tmp = nullptr;
+        const float one = 1.0f;
+        ok = ok && cudaMalloc(&tmp, static_cast<size_t>(N) * K) == cudaSuccess &&
+             cudaMemcpyAsync(w->tensor_scale, &one, sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess &&
+             cudaMemcpyAsync(w->scales_c, scales, n_groups * N * sizeof(uint16_t), cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+             launch_import_int4(codes, static_cast<const uint16_t*>(scales), N, K, group, w->codes, w->scales_t, tmp, w->f8 != 0, st) == cudaSuccess &&
+             cudaStreamSynchronize(st) == cudaSuccess;
+        if (tmp) cudaFree(tmp);
+        ok = ok && finish_int4(w);
     }
     if (!ok) {
         rudder_weight_free(w);
@@ -356,6 +430,7 @@ rudder_status rudder_weight_export(const rudder_weight* w, uint8_t* codes, void*
                                    void* stream)
 {
     if (!w) return RUDDER_ERR_ARG;
+    if (!on_weights_device(w)) return RUDDER_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t n_groups = static_cast<size_t>(w->K / w->G);
     if (w->scheme == RUDDER_W4A4_NVFP4) {
@@ -413,7 +488,7 @@ static rudder_status block_impl(const rudder_block_args* args, int M, const rudd
 {
     if (!args) return RUDDER_ERR_ARG;
     for (int l = 0; l < 4; ++l)
-        if (!args->w[l] || !args->tab[l] || (!args->x[l] && l == 0) || !args->y[l]) return RUDDER_ERR_ARG;
+        if (!args->w[l] || !args->tab[l] || (!args->x[l] && l == 0) || !args->y[l] || !on_weights_device(args->w[l])) return RUDDER_ERR_ARG;
     const size_t need = rudder_block_workspace_bytes(args, M);
     if (!workspace || !aligned(workspace, 256) || workspace_bytes < need || need == 0) return RUDDER_ERR_WORKSPACE;
     // Chained layers (x[l] == NULL, l >= 1) take the previous output through the minimal glue: the V third
@@ -503,6 +578,7 @@ static HostPipe* host_pipe()
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     HostPipe* hp = &g_host_pipe[dev];
+    std::lock_guard<std::mutex> lock(g_state_mutex);
     if (!hp->ready) {
         if (cudaStreamCreateWithFlags(&hp->in, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&hp->out, cudaStreamNonBlocking) != cudaSuccess ||
@@ -598,6 +674,7 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
 {
     if (!w || !X || !codes || !row_scale) return RUDDER_ERR_ARG;
     if (w->scheme == RUDDER_W4A4_NVFP4 && !block_scales) return RUDDER_ERR_ARG;
+    if (!on_weights_device(w)) return RUDDER_ERR_ARG;
     if (M < 1) return RUDDER_ERR_SHAPE;
     SegParams sp;
     rudder_status s = check_table_and_segments(seg, step, tab, M, &sp);
@@ -615,7 +692,11 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
             return RUDDER_ERR_CUDA;
         return RUDDER_OK;
     }
-    if (launch_actq_int(a, qmax_of(w->scheme), false, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    // The kernel writes what production writes for this weight: int8, or (W4A4 on the E4M3 tensor path) the
+    // E4M3 bytes of the same integers, which are then decoded in place so that the caller sees integers.
+    if (launch_actq_int(a, qmax_of(w->scheme), w->f8 != 0, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
+    if (w->f8 != 0 && launch_e4m3_to_int8(static_cast<int8_t*>(codes), static_cast<size_t>(M) * w->K, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     return RUDDER_OK;
 }
@@ -628,6 +709,12 @@ rudder_status rudder_gelu(const uint16_t* X, int64_t ldx, int M, int N, uint16_t
     rudder_status s = ensure_init();
     if (s != RUDDER_OK) return s;
     return launch_gelu(X, ldx, Y, ldy, M, N, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? RUDDER_OK : RUDDER_ERR_CUDA;
+}
+
+rudder_status rudder_selftest_wait_timeout(long long limit_cycles, void* stream)
+{
+    if (limit_cycles < 1000 || limit_cycles > 100000000ll) return RUDDER_ERR_ARG;     // at most ~50 ms of SM clocks
+    return launch_wait_timeout_selftest(limit_cycles, static_cast<cudaStream_t>(stream)) == cudaSuccess ? RUDDER_OK : RUDDER_ERR_CUDA;
 }
 
 rudder_status rudder_device_status(int* last, int* where)

@@ -356,7 +356,7 @@ int gemm_fp4_token_tile(int M, int N)
 {
     if (M <= 128) return 128;
     const long long tiles256 = static_cast<long long>((M + 255) / 256) * ((N + BN_FP4 - 1) / BN_FP4);
-    return tiles256 >= 148 ? 256 : 128;
+    return tiles256 >= device_sm_count() ? 256 : 128;
 }
 int gemm_fp4_store_rows(int M, int N) { return gemm_fp4_token_tile(M, N) / 4; }
 

@@ -332,11 +332,7 @@ gemm_nvfp4_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_co
 // The pair kernel needs whole 256-channel tiles and is worth its fixed cost only with many tokens.
 bool gemm_fp4_use_pair(int M, int N, int K)
 {
-#ifdef RUDDER_NO_PAIR
-    return false;
-#else
     return M >= 1024 && N % 256 == 0 && K % 256 == 0;
-#endif
 }
 
 static int g_pair_clusters[64] = {0};
@@ -350,7 +346,7 @@ cudaError_t gemm_fp4_pair_init()
     if (dev >= 0 && dev < 64) {
         // how many CTA pairs the device runs at once
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * 148, 1, 1);
+        cfg.gridDim = dim3(2 * device_sm_count(), 1, 1);
         cfg.blockDim = dim3(fp4::NUM_THREADS, 1, 1);
         cfg.dynamicSmemBytes = fp4::PAIR_DYN_SMEM;
         int n = 0;

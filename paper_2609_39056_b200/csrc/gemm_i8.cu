@@ -66,18 +66,9 @@ namespace {
 
 constexpr int BN = 128;          // output channels per tile (MMA M)
 constexpr int KSTAGE = 128;      // input channels (= bytes of int8 per row) per pipeline stage
-#ifndef RUDDER_PSX
-#define RUDDER_PSX 3             // persistent form: activation stages
-#endif
-#ifndef RUDDER_PSW
-#define RUDDER_PSW 3             // persistent form: unpacked-weight stages
-#endif
-#ifndef RUDDER_PERSIST_MIN_TILES
-#define RUDDER_PERSIST_MIN_TILES (3 * 148)   // fewest tiles for which the persistent form is used
-#endif
-#ifndef RUDDER_PERSIST_MIN_G
-#define RUDDER_PERSIST_MIN_G 0   // (build-time switch: a huge value turns the persistent form off)
-#endif
+constexpr int kPersistStagesX = 3;   // persistent form: activation stages
+constexpr int kPersistStagesW = 3;   // persistent form: unpacked-weight stages
+constexpr int kPersistTilesPerSm = 3;   // fewest tiles per SM for which the persistent form is used
 constexpr int W_BYTES = BN * KSTAGE;
 constexpr int SR = 4;            // packed-weight stages (256-token tiles)
 constexpr int RAW_BYTES = BN * KSTAGE / 2;
@@ -102,8 +93,8 @@ constexpr int RUDDER_SLEEP_EPI = 0;
 // of 128 tokens x 128 channels of bf16 output gets its own shared memory (the rings belong to the next
 // tile by the time a tile is written), paid for with shallower rings.
 template <int TT, bool PERSIST = false> struct Tile {
-    static constexpr int SX = PERSIST ? RUDDER_PSX : ((TT == 256) ? 4 : 8);
-    static constexpr int SW = PERSIST ? RUDDER_PSW : 4;  // unpacked-weight stages
+    static constexpr int SX = PERSIST ? kPersistStagesX : ((TT == 256) ? 4 : 8);
+    static constexpr int SW = PERSIST ? kPersistStagesW : 4;  // unpacked-weight stages
     static constexpr int X_BYTES = TT * KSTAGE;
     static constexpr int OFF_X = 0;
     static constexpr int OFF_W = OFF_X + SX * X_BYTES;
@@ -619,7 +610,8 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
             for (int pass = 0; pass < 2; ++pass) {
                 if (threadIdx.x == 256) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+                // the barrier also makes the verdict common to all drain threads: they leave the tile loop together
+                ok = bar_sync_and(1, EPI_THREADS, ok);
                 if (ok) {
                     if (ch_local < p.out_pitch) {
                         const uint32_t step = static_cast<uint32_t>(p.out_pitch) * 2u;
@@ -806,17 +798,14 @@ static cudaError_t launch_one(const GemmI8Args& a, const GemmI8Plan& plan, cudaS
 GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool f8, bool dump)
 {
     GemmI8Plan plan;
+    const int sm_count = device_sm_count();
     // The persistent form pays where the drain warps have slack during the main loop and a CTA gets
     // several tiles: one scale per output channel (a single group per tile, drain warps idle: 20 % faster)
     // and groups of 128 on the integer path (6 %); level at groups of 64, 10 % slower on the E4M3 path.
     {
         const long long tiles = static_cast<long long>((M + 255) / 256) * ((N + BN - 1) / BN);
-#ifdef RUDDER_PERSIST_ANY_G
-        const bool shape_ok = true;
-#else
         const bool shape_ok = G >= K || (G >= 128 && !f8);
-#endif
-        plan.persist = !dump && M > 256 && shape_ok && G >= RUDDER_PERSIST_MIN_G && tiles >= RUDDER_PERSIST_MIN_TILES;
+        plan.persist = !dump && M > 256 && shape_ok && tiles >= static_cast<long long>(kPersistTilesPerSm) * sm_count;
     }
     plan.token_tile = M > 256 ? 256 : (M > 32 ? 64 : 32);    // up to 256 tokens: small tiles, eight TMEM buffers
     plan.splitk = 1;
@@ -827,7 +816,7 @@ GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool f8, bool dump)
     const int base = m_tiles * n_tiles;
     const size_t m_pad = static_cast<size_t>(m_tiles) * plan.token_tile;
     int sk = 1;
-    while (sk < 16 && base * (sk * 2) <= 160 && (K / KSTAGE) % (sk * 2) == 0 && K / (sk * 2) >= 2 * KSTAGE &&
+    while (sk < 16 && base * (sk * 2) <= sm_count + sm_count / 12 && (K / KSTAGE) % (sk * 2) == 0 && K / (sk * 2) >= 2 * KSTAGE &&
            static_cast<size_t>(sk * 2) * N * m_pad * sizeof(float) <= (size_t(2) << 20))
         sk *= 2;
     plan.splitk = sk;

@@ -62,16 +62,25 @@ struct ActqArgs {
     SegParams seg;
 };
 
+// SMs of the current device (cached per device).  The one number every tile / split / grid choice below is
+// derived from, so that workspace sizing, tensor-map boxes and launches always see the same plan.
+int device_sm_count();
+
 // ---- launches (each returns cudaGetLastError of its launch) ----------------------------------
 cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G, uint8_t* codes_il,
                              float* scales_t, uint16_t* scales_c, float* dinv, int8_t* tmp_codes, bool signmag,
                              cudaStream_t st);
+cudaError_t launch_import_int4(const uint8_t* canonical, const uint16_t* scales_c, int N, int K, int G, uint8_t* codes_il,
+                               float* scales_t, int8_t* tmp_codes, bool signmag, cudaStream_t st);
+cudaError_t launch_import_nvfp4_scales(const uint8_t* sb_canonical, int N, int K, uint8_t* sf_tiled, size_t sf_tiled_bytes, cudaStream_t st);
 cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, bool signmag, cudaStream_t st);
 
 cudaError_t launch_gelu(const uint16_t* X, int64_t ldx, uint16_t* Y, int64_t ldy, int M, int N, int sm_count, cudaStream_t st);
 cudaError_t actq_init();
+cudaError_t launch_wait_timeout_selftest(long long limit_cycles, cudaStream_t st);
 // e4m3: the codes (integers in [-7, 7]) are written as E4M3 bytes for the FP8 tensor path instead of int8
 cudaError_t launch_actq_int(const ActqArgs& a, int qmax, bool e4m3, int8_t* codes, int64_t ldc, float* r, cudaStream_t st);
+cudaError_t launch_e4m3_to_int8(int8_t* codes, size_t n_bytes, cudaStream_t st);   // parity hook: E4M3 bytes -> the integers they hold, in place
 cudaError_t launch_actq_nvfp4(const ActqArgs& a, uint8_t* codes, uint8_t* sf, bool sf_tiled, float* r, cudaStream_t st);
 cudaError_t launch_pack_nvfp4(const float* W, const float* d, int N, int K, uint8_t* codes, uint8_t* sb_canonical,
                               uint8_t* sf_tiled, size_t sf_tiled_bytes, float* dinv, float* tensor_scale,

@@ -158,6 +158,44 @@ cudaError_t launch_pack_int4(const float* W, const float* d, int N, int K, int G
     return cudaGetLastError();
 }
 
+// ---- import of a canonical packed weight (the layout rudder_weight_export writes) -------------------
+// canonical nibbles [N, K/2] (low nibble = even k, two's complement) -> one int8 code per byte [N, K]
+__global__ void import_int4_expand_kernel(const uint8_t* __restrict__ canonical, size_t total, int8_t* __restrict__ q)
+{
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const uint8_t b = canonical[idx];
+    const int lo = b & 0xF, hi = b >> 4;
+    q[2 * idx] = static_cast<int8_t>(lo > 7 ? lo - 16 : lo);
+    q[2 * idx + 1] = static_cast<int8_t>(hi > 7 ? hi - 16 : hi);
+}
+// fp16 scales [N, K/G] -> the GEMM's fp32 [K/G, N] = Delta_W / 16
+__global__ void import_scales_kernel(const uint16_t* __restrict__ scales_c, int N, int n_groups, float* __restrict__ scales_t)
+{
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= static_cast<size_t>(N) * n_groups) return;
+    const int j = static_cast<int>(idx / n_groups), g = static_cast<int>(idx % n_groups);
+    scales_t[static_cast<size_t>(g) * N + j] = __half2float(__ushort_as_half(scales_c[idx])) * 0.0625f;
+}
+
+cudaError_t launch_import_int4(const uint8_t* canonical, const uint16_t* scales_c, int N, int K, int G, uint8_t* codes_il,
+                               float* scales_t, int8_t* tmp_codes, bool signmag, cudaStream_t st)
+{
+    const size_t total = static_cast<size_t>(N) * (K / 2);
+    import_int4_expand_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(canonical, total, tmp_codes);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (signmag)
+        pack_int4_signmag_kernel<<<static_cast<unsigned>((total / 4 + 255) / 256), 256, 0, st>>>(tmp_codes, N, K, reinterpret_cast<uint32_t*>(codes_il));
+    else
+        pack_int4_interleave_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(tmp_codes, N, K, codes_il);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t ns = static_cast<size_t>(N) * (K / G);
+    import_scales_kernel<<<static_cast<unsigned>((ns + 255) / 256), 256, 0, st>>>(scales_c, N, K / G, scales_t);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, bool signmag, cudaStream_t st)
 {
     const size_t total = static_cast<size_t>(N) * (K / 2);

@@ -44,6 +44,25 @@ __global__ void nvfp4_quantize_kernel(const float* __restrict__ W, const float* 
     sf_tiled[nvfp4_sf_offset(j, b, K / 64)] = static_cast<uint8_t>(sb);
 }
 
+// Import: row-major UE4M3 block scales [N, K/16] -> the tensor core's tiled order (padding rows stay zero).
+__global__ void nvfp4_tile_scales_kernel(const uint8_t* __restrict__ sb_canonical, int N, int K, uint8_t* __restrict__ sf_tiled)
+{
+    const int n_blocks = K / 16;
+    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= static_cast<size_t>(N) * n_blocks) return;
+    const int j = static_cast<int>(idx / n_blocks), b = static_cast<int>(idx % n_blocks);
+    sf_tiled[nvfp4_sf_offset(j, b, K / 64)] = sb_canonical[idx];
+}
+
+cudaError_t launch_import_nvfp4_scales(const uint8_t* sb_canonical, int N, int K, uint8_t* sf_tiled, size_t sf_tiled_bytes, cudaStream_t st)
+{
+    cudaError_t e = cudaMemsetAsync(sf_tiled, 0, sf_tiled_bytes, st);
+    if (e != cudaSuccess) return e;
+    const size_t total = static_cast<size_t>(N) * (K / 16);
+    nvfp4_tile_scales_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(sb_canonical, N, K, sf_tiled);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pack_nvfp4(const float* W, const float* d, int N, int K, uint8_t* codes, uint8_t* sb_canonical,
                               uint8_t* sf_tiled, size_t sf_tiled_bytes, float* dinv, float* tensor_scale,
                               unsigned int* amax_bits, cudaStream_t st)

@@ -49,8 +49,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  `abort_word` is a shared int: non-zero means some role of this CTA gave up.
 // `sleep_ns` > 0: back off between polls so that a waiting warp does not take issue slots from the
 // warps that share its scheduler.
+// `limit_cycles`: how long the wait may last (the default of about a second is far beyond any wait of a
+// healthy kernel; the self-test passes a short one).
 template <int SLEEP_NS = 0>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int where) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int where,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();          // SM-local cycle counter: cheap to read
     for (uint32_t it = 1;; ++it) {
@@ -58,13 +61,31 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 0u) {
             if (*abort_word != 0) return false;
-            if (clock64() - t0 > kWaitLimitCycles) break;
+            if (clock64() - t0 > limit_cycles) break;
         }
     }
     *abort_word = where;
     atomicExch(&g_device_status[1], where);
     atomicExch(&g_device_status[0], 7);   // RUDDER_ERR_TIMEOUT
     return false;
+}
+
+// Named barrier over `count` threads that also ANDs a predicate across them: every participant gets the
+// same verdict, so a role that gave up a bounded wait takes the whole group out of its loop together
+// (a thread that left alone would strand the others at their next barrier).
+__device__ __forceinline__ bool bar_sync_and(int id, int count, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}\n"
+        : "=r"(r)
+        : "r"(static_cast<uint32_t>(pred)), "r"(id), "r"(count)
+        : "memory");
+    return r != 0;
 }
 
 // ---- register reallocation between warpgroups (all 4 warps of a warpgroup execute it together) ----

@@ -21,6 +21,7 @@ rudder_status static_workspace(void** out)
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RUDDER_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_state_mutex);
     if (g_static_workspace_addr[dev] == nullptr) {
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || ptr == nullptr) return RUDDER_ERR_CUDA;

@@ -53,3 +53,15 @@ def test_linear_rejects_null_and_workspace_query(L):
     assert L.rudder_linear_workspace_bytes(None, 16) == 0
     assert L.rudder_block(None, 1, None, 0, None, 0, None) == rd.ERR_ARG
     assert L.rudder_weight_free(None) == rd.OK
+
+
+def test_import_rejects_bad_arguments_on_host(L):
+    import paper_2609_39056_b200 as rd
+    out = ctypes.c_void_p()
+    fake = ctypes.c_void_p(0x1000)      # never dereferenced: the checks below fail first
+    f = L.rudder_weight_import
+    assert f(None, fake, fake, None, 128, 128, rd.W4A8_INT, 64, None, ctypes.byref(out)) == rd.ERR_ARG
+    assert f(fake, fake, fake, None, 128, 256, rd.W4A4_NVFP4, 16, None, ctypes.byref(out)) == rd.ERR_ARG   # NVFP4 needs its tensor scale
+    assert f(fake, fake, fake, None, 100, 128, rd.W4A8_INT, 64, None, ctypes.byref(out)) == rd.ERR_SHAPE
+    assert f(fake, fake, fake, None, 128, 256, rd.W4A8_INT, 32, None, ctypes.byref(out)) == rd.ERR_SHAPE
+    assert out.value is None

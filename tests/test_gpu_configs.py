@@ -75,14 +75,15 @@ def run_block_config(rd, cfg, steps, n_random):
 
 
 def test_config2_w4a8_block_full_size(rd):
-    """Configuration 2: hidden 2048, MLP 8192, 4096 + 64 + 256 tokens, W4A8 group 64, steps 0 and 9."""
-    run_block_config(rd, wl.config(2), steps=(0, 9), n_random=24)
+    """Configuration 2: hidden 2048, MLP 8192, 4096 + 64 + 256 tokens, W4A8 group 64, steps 0, 4 and 9."""
+    run_block_config(rd, wl.config(2), steps=(0, 4, 9), n_random=256)
 
 
 @pytest.mark.parametrize("scheme", ["w4a4", "nvfp4"])
 def test_config3_w4a4_block_full_size(rd, scheme):
-    """Configuration 3: hidden 3072, MLP 12288, batch 2 x (8192 + 64 + 512) tokens, step 7."""
-    run_block_config(rd, wl.config(3, scheme), steps=(7,), n_random=12)
+    """Configuration 3: hidden 3072, MLP 12288, batch 2 x (8192 + 64 + 512) tokens; steps 0, 7 and 9 on
+    256 seeded rows plus every segment's first and last row and the rows around tile edges."""
+    run_block_config(rd, wl.config(3, scheme), steps=(0, 7, 9), n_random=256)
 
 
 @pytest.mark.parametrize("scheme", ["w4a8", "w4a4"])

@@ -1,14 +1,16 @@
 """rudder_linear_static: the entry point for callers that cannot allocate device memory (code inside
 a captured or real-time region, plug-ins that only receive input and output buffers).  Its scratch
 is a fixed array inside the library, so the test checks it against rudder_linear, whose scratch the
-caller allocates: same kernels, so the outputs must agree within the suite's tolerance (they are in
-fact identical), on two calls in a row that reuse the array, and an oversized request is refused."""
+caller allocates (same kernels, so the outputs must agree within the suite's tolerance -- they are in
+fact identical) and against the CPU oracle, on two calls in a row that reuse the array; an oversized
+request is refused."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import workloads as wl
-from helpers import ABS_TOL, REL_TOL, GpuLinear, bf16_to_np
+from helpers import ABS_TOL, REL_TOL, GpuLinear, bf16_to_np, check_output
 
 pytestmark = pytest.mark.gpu
 
@@ -35,6 +37,11 @@ def test_static_workspace_entry_point_matches_rudder_linear():
         torch.cuda.synchronize()
         assert _close(got, want)
         assert torch.equal(got, want)
+        # and against the CPU oracle, like every other entry point
+        inp = g.inp
+        ref = oracle.rudder_linear(inp.X_bf16, oracle.pack_int4(inp.W, inp.d, g.group), inp.gamma, None, step,
+                                   oracle.RANGE_PER_TOKEN, inp.seg_offsets, inp.seg_stream, g.scheme, inp.bias)
+        check_output(bf16_to_np(got), ref["y64"])
     # and the first shape again, after the array was overwritten by the second
     want = rd.rudder_linear(first.w, first.X, first.seg, 0, first.tab, first.bias)
     got = torch.empty_like(want)
