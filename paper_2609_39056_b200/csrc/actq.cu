@@ -283,6 +283,7 @@ __global__ void __launch_bounds__(256) actq_nvfp4_kernel(ActqArgs a, int M_pad, 
 // integer max instruction for the range (non-negative floats order like their bit patterns), a
 // shared-memory atomic max across warps, and a table for the reciprocal of the block scale.
 constexpr int kRowSlots = 4;
+constexpr int kFewRows = 256;                      // up to this many rows the integer prologue runs one CTA per row
 constexpr int W_ROW_FULL = 40;                     // wait identifier reported on a timeout
 
 struct RowOut {
@@ -400,6 +401,77 @@ __device__ __forceinline__ uint2 e4m3x8(const f32x2* v, float qmaxf) {
         h[i] = e4m3x2(lo, hi);
     }
     return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+}
+
+// ---- few rows (up to 256): one CTA per row ---------------------------------------------------------
+// With a handful of rows the prologue is pure latency, so it is kept to one round trip: the 256 threads
+// of a CTA load the whole row at once (NP 16-byte pieces each, rows up to 2048 NP channels), the range
+// is reduced through shared memory with one barrier, the codes are rounded from the registers.  The
+// arithmetic is the packed two-lane form of the row kernel (mul_dinv8, s8x8, e4m3x8): the very device
+// functions the fused small-M GEMM quantises with, so this kernel doubles as its parity hook.
+template <int NP>
+__global__ void __launch_bounds__(256) actq_int_cta_row_kernel(ActqArgs a, int qmax, int e4m3, int8_t* __restrict__ codes, int64_t ldc,
+                                                                float* __restrict__ r)
+{
+    __shared__ uint32_t wmax[8];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the GEMM behind this kernel may start its set-up
+    asm volatile("griddepcontrol.wait;" ::: "memory");                // X may come from the kernel before this one
+    const int row = blockIdx.x;
+    const int t = threadIdx.x;
+    if (row == 0 && a.zero_ints != nullptr)
+        for (int i = t; i < a.n_zero; i += 256) a.zero_ints[i] = 0;
+    const float g = a.gamma_step[stream_of_row(a.seg, row)];
+    const uint4* xrow = reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(row) * a.ldx);
+    const float4* dv = reinterpret_cast<const float4*>(a.dinv);
+    const int n_chunks = a.K >> 3;
+    uint4 xr[NP];
+    f32x2 dd[NP][4];
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        const int c = t + i * 256;
+        if (c < n_chunks) {
+            xr[i] = ld_nc_16(xrow + c);
+            const float4 d0 = __ldg(dv + 2 * c), d1 = __ldg(dv + 2 * c + 1);
+            dd[i][0] = pack2(d0.x, d0.y); dd[i][1] = pack2(d0.z, d0.w); dd[i][2] = pack2(d1.x, d1.y); dd[i][3] = pack2(d1.z, d1.w);
+        }
+    }
+    float range;
+    if (a.clip_step == nullptr) {
+        float amax = 0.0f;                         // max |x dinv|; the gain is applied to the maximum (monotonic rounding, gamma > 0)
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            if (t + i * 256 < n_chunks) {
+                f32x2 u[4];
+                amax = fmaxf(amax, mul_dinv8(xr[i], dd[i], u));
+            }
+        }
+        const uint32_t wm = __reduce_max_sync(0xffffffffu, __float_as_uint(amax));
+        if ((t & 31) == 0) wmax[t >> 5] = wm;
+        __syncthreads();
+        uint32_t m = wmax[0];
+#pragma unroll
+        for (int i = 1; i < 8; ++i) m = max(m, wmax[i]);
+        range = __fmul_rn(__uint_as_float(m), g);
+    } else {
+        range = *a.clip_step;
+    }
+    const float qmaxf = static_cast<float>(qmax);
+    const float inv = (range != 0.0f) ? __fdiv_rn(qmaxf, range) : 0.0f;
+    const f32x2 g2 = pack2(g, g), inv2 = pack2(inv, inv);
+    const bool clamp = a.clip_step != nullptr;
+    uint2* crow = reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldc);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        const int c = t + i * 256;
+        if (c < n_chunks) {
+            f32x2 u[4];
+            mul_dinv8(xr[i], dd[i], u);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { mul2(u[k], g2); mul2(u[k], inv2); }
+            crow[c] = e4m3 ? e4m3x8(u, qmaxf) : (clamp ? s8x8<true>(u, qmaxf) : s8x8<false>(u, qmaxf));
+        }
+    }
+    if (t == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, static_cast<float>(qmax)), g) : 0.0f;
 }
 
 template <bool FP4, int NCH>
@@ -669,6 +741,15 @@ cudaError_t launch_actq_int(const ActqArgs& a, int qmax, bool e4m3, int8_t* code
     RowOut o;
     o.codes = codes; o.ldc = ldc; o.sf = nullptr; o.sf_tiled = 0; o.r = r; o.M_pad = a.M; o.qmax = qmax; o.e4m3 = e4m3 ? 1 : 0;
     cudaError_t err = cudaSuccess;
+    const bool aligned16 = (reinterpret_cast<uintptr_t>(a.X) % 16 == 0) && ((a.ldx * 2) % 16 == 0) &&
+                           (reinterpret_cast<uintptr_t>(codes) % 8 == 0) && (ldc % 8 == 0) && (a.K % 8 == 0);
+    if (a.M <= kFewRows && a.K <= 8192 && aligned16) {
+        // few rows: one CTA per row, one round trip
+        if (a.K <= 2048)      err = launch_early(actq_int_cta_row_kernel<1>, a.M, 256, 0, st, a, qmax, e4m3 ? 1 : 0, codes, ldc, r);
+        else if (a.K <= 4096) err = launch_early(actq_int_cta_row_kernel<2>, a.M, 256, 0, st, a, qmax, e4m3 ? 1 : 0, codes, ldc, r);
+        else                  err = launch_early(actq_int_cta_row_kernel<4>, a.M, 256, 0, st, a, qmax, e4m3 ? 1 : 0, codes, ldc, r);
+        return err != cudaSuccess ? err : cudaGetLastError();
+    }
     if (!launch_row<false>(a, o, a.M, st, &err)) {
         const int blocks = (a.M * 32 + 255) / 256;         // unaligned or very long rows: one warp per row, row read twice
         if (a.zero_ints != nullptr && cudaMemsetAsync(a.zero_ints, 0, sizeof(int) * a.n_zero, st) != cudaSuccess) return cudaErrorUnknown;

@@ -211,6 +211,19 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
 
     int8_t* codes = static_cast<int8_t*>(workspace);
     float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
+    if (gemm_i8_fewrows_applies(M, w->N, w->K, w->G)) {
+        // A handful of rows: the light prologue (int8 codes, whatever the weight layout) and the register-level GEMM.
+        if (launch_actq_int(a, qmax_of(w->scheme), false, codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        GemmI8FewRowsArgs f;
+        f.codes = codes; f.ldc = w->K; f.row_scale = r; f.wq = w->codes; f.signmag = w->f8 != 0;
+        f.w_scales_t = w->scales_t; f.bias = bias; f.Y = Y; f.ldy = ldy;
+        f.M = M; f.N = w->N; f.K = w->K; f.G = w->G;
+        f.acc = acc; f.row0 = row0; f.rows = rows; f.col0 = col0; f.cols = cols;
+        if (launch_gemm_i8_fewrows(f, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        return RUDDER_OK;
+    }
     const GemmI8Plan plan = gemm_i8_plan(M, w->N, w->K, w->G, w->f8 != 0, acc != nullptr);
     GemmI8Args g;
     g.partials = nullptr; g.counters = nullptr;
@@ -694,9 +707,10 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
     }
     // The kernel writes what production writes for this weight: int8, or (W4A4 on the E4M3 tensor path) the
     // E4M3 bytes of the same integers, which are then decoded in place so that the caller sees integers.
-    if (launch_actq_int(a, qmax_of(w->scheme), w->f8 != 0, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    const bool e4m3 = w->f8 != 0 && !gemm_i8_fewrows_applies(M, w->N, w->K, w->G);     // the few-rows GEMM reads int8 whatever the weight layout
+    if (launch_actq_int(a, qmax_of(w->scheme), e4m3, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
-    if (w->f8 != 0 && launch_e4m3_to_int8(static_cast<int8_t*>(codes), static_cast<size_t>(M) * w->K, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    if (e4m3 && launch_e4m3_to_int8(static_cast<int8_t*>(codes), static_cast<size_t>(M) * w->K, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     return RUDDER_OK;
 }

@@ -138,4 +138,20 @@ size_t gemm_i8_scratch_bytes(int M, int N, int K, bool dump, size_t* counters_of
 cudaError_t launch_gemm_i8(const GemmI8Args& a, cudaStream_t st);
 cudaError_t gemm_i8_init();     // one-time function attributes (dynamic shared memory opt-in)
 
+// Few rows (action / proprio-only passes): register-level GEMM after the prologue kernel, see gemm_i8_fewrows.cu.
+struct GemmI8FewRowsArgs {
+    const int8_t* codes; int64_t ldc;   // Q_X int8 [M, ldc]
+    const float* row_scale;             // r [M]
+    const uint8_t* wq;                  // packed weights
+    bool signmag;                       // weights in the sign-magnitude layout (W4A4 with groups up to 128)
+    const float* w_scales_t;
+    const float* bias;
+    uint16_t* Y; int64_t ldy;
+    int M, N, K, G;
+    int32_t* acc;                       // accumulator dump (parity hook) or nullptr
+    int row0, rows, col0, cols;
+};
+bool gemm_i8_fewrows_applies(int M, int N, int K, int G);
+cudaError_t launch_gemm_i8_fewrows(const GemmI8FewRowsArgs& a, cudaStream_t st);
+
 }  // namespace rudder

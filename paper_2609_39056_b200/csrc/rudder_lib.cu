@@ -7,6 +7,7 @@
 #include "pack_nvfp4.cu"
 #include "actq.cu"
 #include "gemm_i8.cu"
+#include "gemm_i8_fewrows.cu"
 #include "gemm_fp4.cu"
 #include "gemm_fp4_pair.cu"
 #include "glue.cu"
