@@ -386,6 +386,47 @@ def small_m_sweep(rd, torch, dev, pk, schemes=("w4a8", "w4a4"), sizes=(2048, 409
     return out
 
 
+def crossattn_kv(rd, torch, dev, pk, schemes=("w4a8", "w4a4", "nvfp4")):
+    """The cross-attention key / value projections (one global-text region each): both linears of one step in a CUDA
+    graph over the 10 steps of tables, microseconds per pair, cuBLAS BF16 on the same shapes beside it."""
+    out = []
+    for scheme in schemes:
+        cfg = wl.config(5, scheme)
+        lins = cfg.draw()
+        items = []
+        for l in lins:
+            W = torch.from_numpy(l.W).to(dev)
+            d = torch.from_numpy(l.d).to(dev)
+            w = rd.rudder_pack_weights(W, d, rd.SCHEMES[scheme], cfg.group)
+            items.append(dict(w=w, tab=rd.ScaleTable(torch.from_numpy(l.gamma).to(dev), None, rd.RANGE_PER_TOKEN),
+                              X=torch.from_numpy(l.X_bf16.view(np.int16)).to(dev).view(torch.bfloat16), bias=torch.from_numpy(l.bias).to(dev),
+                              Y=torch.empty((l.M, l.N), dtype=torch.bfloat16, device=dev),
+                              ws=torch.empty(rd.rudder_linear_workspace_bytes(w, l.M) + 256, dtype=torch.uint8, device=dev),
+                              Wb=torch.randn((l.N, l.K), dtype=torch.bfloat16, device=dev)))
+        seg = rd.Segments(lins[0].seg_offsets, lins[0].seg_stream)
+        stream = torch.cuda.Stream()
+
+        def pair(t):
+            for it in items:
+                rd.rudder_linear(it["w"], it["X"], seg, t, it["tab"], it["bias"], Y=it["Y"], workspace=it["ws"])
+
+        def pair_bf16():
+            for it in items:
+                torch.matmul(it["X"], it["Wb"].t(), out=it["Y"])
+
+        with torch.cuda.stream(stream):
+            for t in range(3):
+                pair(t)
+                pair_bf16()
+            stream.synchronize()
+        us = _graph_us(torch, stream, [(lambda t=t: pair(t)) for t in range(cfg.T)])
+        us_b = _graph_us(torch, stream, [pair_bf16 for _ in range(cfg.T)])
+        ops = cfg.ops()
+        out.append({"workload": cfg.name, "scheme": scheme, "us_per_pair": us, "tops": ops / (us * 1e-6) / 1e12,
+                    "us_bf16_cublas": us_b, "x_bf16": us_b / us})
+    return out
+
+
 def calibrator_timing(rd, torch, dev):
     """Toy calibrator (Eq. 9) on the QKV layer of configuration 2, one layer-step: wall time of the whole
     search (every candidate is one static-mode rudder_linear plus the error reduction)."""
@@ -520,6 +561,7 @@ def run_ours(args):
             del m2
             torch.cuda.empty_cache()
         also["cfg4_small_m_sweep"] = small_m_sweep(rd, torch, dev, pk)
+        also["cfg5_crossattn_kv"] = crossattn_kv(rd, torch, dev, pk)
         also["toy_calibrator"] = calibrator_timing(rd, torch, dev)
     if sampler is not None:
         sampler.stop()
@@ -556,7 +598,7 @@ def make_summary(cfg, sustained, roofline, bf16_ms, also):
     peak, of the nominal dense peak, speed-up over cuBLAS BF16]; per small-M point [us per linear, fraction of
     the measured HBM bandwidth, speed-up over cuBLAS BF16]."""
     r3 = lambda v: None if v is None else float(f"{v:.3g}")
-    out = {"keys": "block: [ms_sustained, TOPS, gemm_frac_sustained_peak, gemm_frac_nominal, x_bf16]; cfg4: {scheme_K: {M: [us, hbm_frac, x_bf16]}}"}
+    out = {"keys": "block: [ms_sustained, TOPS, gemm_frac_sustained_peak, gemm_frac_nominal, x_bf16]; cfg4: {scheme_K: {M: [us, hbm_frac, x_bf16]}}; cfg5: {scheme: [us_per_kv_pair, TOPS, x_bf16]}"}
     tag = lambda name: name.split("_block")[0] + name.split("m4416")[-1].split("m17536")[-1]
     out[tag(cfg.name)] = [r3(sustained["ms_per_step"]), r3(sustained["tops"]), r3(roofline["frac"]), r3(roofline["frac_of_nominal_dense"]),
                           r3(bf16_ms / sustained["ms_per_step"]) if bf16_ms else None]
@@ -570,6 +612,9 @@ def make_summary(cfg, sustained, roofline, bf16_ms, also):
         for r in sweep:
             c4.setdefault(f"{r['scheme']}_{r['K']}", {})[str(r["M"])] = [r3(r["us_per_linear"]), r3(r["hbm_frac"]), r3(r.get("x_bf16"))]
         out["cfg4"] = c4
+    ca = (also or {}).get("cfg5_crossattn_kv")
+    if ca:
+        out["cfg5_crossattn_kv"] = {r["scheme"]: [r3(r["us_per_pair"]), r3(r["tops"]), r3(r["x_bf16"])] for r in ca}
     return out
 
 

@@ -182,6 +182,25 @@ size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M);
 rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
                            void* workspace, size_t workspace_bytes, void* stream);
 
+/* rudder_block_dit -- the same four linears wired as one DiT block with its BF16 glue (normalisation, GELU and
+ * residual additions stay in BF16: Appendix "Quantization"), run end to end on the device from x[0] alone:
+ *     h   = x + O( V-third of QKV( rmsnorm(x; norm1_weight) ) )      [the V third stands in for attention, which stays outside]
+ *     out = h + down( gelu( up( rmsnorm(h; norm2_weight) ) ) )
+ * args->x[0] is the block input [M, H]; args->x[1..3] must be NULL; args->y[l] still receive the four linears' outputs;
+ * shapes must be QKV H -> 3H, O H -> H, up H -> F, down F -> H (else RUDDER_ERR_SHAPE).  glue->out [M, ldout] receives
+ * the block output.  Workspace: rudder_block_dit_workspace_bytes(args, M), 256-byte aligned.
+ * rmsnorm, gelu and the additions are the bit-defined forms of rudder_rmsnorm, rudder_gelu and rudder_add below. */
+typedef struct {
+    const float* norm1_weight;   /* [H] fp32, 16-byte aligned */
+    const float* norm2_weight;   /* [H] fp32, 16-byte aligned */
+    float eps;                   /* >= 0 */
+    uint16_t* out;               /* bf16 [M, ldout] */
+    int64_t ldout;
+} rudder_block_glue;
+size_t rudder_block_dit_workspace_bytes(const rudder_block_args* args, int M);
+rudder_status rudder_block_dit(const rudder_block_args* args, const rudder_block_glue* glue, int M, const rudder_segments* seg,
+                               int step, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Measurement hook: rudder_block with a CUDA event between consecutive kernels.  ms (HOST [8])
  * receives the device time of each launch in order: prologue and GEMM of QKV, O, up, down.
  * Creates and destroys its events and SYNCHRONISES the stream before returning. */
@@ -230,6 +249,17 @@ rudder_status rudder_linear_dump_acc(const rudder_weight* w, const uint16_t* X, 
  * rounded to nearest on its own (no fused multiply-add): the result is defined bit for bit.
  * X, Y bf16 [M, ld]; N % 8 == 0; 16-byte aligned pointers, leading dimensions multiples of 8. */
 rudder_status rudder_gelu(const uint16_t* X, int64_t ldx, int M, int N, uint16_t* Y, int64_t ldy, void* stream);
+
+/* BF16 RMS normalisation of every row with a weight per channel (which normalisation the paper's models use is not
+ * stated; reading: RMSNorm): Y = bf16((x * r) * weight), r = 1 / sqrt(mean(x^2) + eps).  Defined bit for bit: fp32, one
+ * warp per row, lane l adds x * x (product and sum rounded separately) of the 8-value pieces l, l + 32, ... in order; the
+ * 32 partial sums are combined by the exchange l ^ 16, 8, 4, 2, 1; mean = sum / N, r by IEEE division and square root.
+ * X, Y bf16 [M, ld], weight fp32 [N]; N % 8 == 0; 16-byte aligned pointers, leading dimensions multiples of 8. */
+rudder_status rudder_rmsnorm(const uint16_t* X, int64_t ldx, int M, int N, const float* weight, float eps, uint16_t* Y, int64_t ldy,
+                             void* stream);
+/* BF16 residual addition, elementwise: Y = bf16(A + B), one fp32 addition.  Same shape and alignment rules. */
+rudder_status rudder_add(const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, int M, int N, uint16_t* Y, int64_t ldy,
+                         void* stream);
 
 /* Reads and clears the device status word (SYNCHRONISES the device).  *last (HOST) receives
  * RUDDER_OK or RUDDER_ERR_TIMEOUT; *where (HOST, may be NULL) a code naming the wait that gave up. */

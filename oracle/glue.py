@@ -1,4 +1,4 @@
-"""CPU oracle of the BF16 glue of a chained block: GELU (TEST INFRASTRUCTURE ONLY).
+"""CPU oracle of the BF16 glue of a chained block: GELU, RMS normalisation, residual add (TEST INFRASTRUCTURE ONLY).
 
 The paper keeps GELU in BF16 and does not say which GELU.  Reading: the tanh form
     gelu(x) = x/2 (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3)))
@@ -55,3 +55,37 @@ def gelu_f32(x):
 def gelu_bf16(bits):
     """bf16 bit patterns in -> bf16 bit patterns out."""
     return f32_to_bf16(gelu_f32(bf16_to_f32(bits)))
+
+
+def rmsnorm_bf16(bits, weight, eps):
+    """RMS normalisation of every row: y = bf16((x r) w), r = 1 / sqrt(mean(x^2) + eps), in the fixed fp32 order
+    that makes the result (and the integer codes the next layer makes of it) a matter of definition, not of
+    summation order: the row is cut into pieces of 8 values; partial sum l (of 32) adds x*x of pieces l, l + 32,
+    ... in order, product and sum rounded separately; the partials are combined pairwise l ^ 16, 8, 4, 2, 1."""
+    x = bf16_to_f32(bits)
+    M, N = x.shape
+    assert N % 8 == 0
+    w = np.asarray(weight, dtype=np.float32)
+    chunks = N // 8
+    rounds = (chunks + 31) // 32
+    xp = np.zeros((M, rounds * 32 * 8), np.float32)
+    xp[:, :N] = x                                             # padding adds +0.0: no effect on any partial sum
+    xp = xp.reshape(M, rounds, 32, 8)
+    acc = np.zeros((M, 32), np.float32)
+    for j in range(rounds):
+        for e in range(8):
+            v = xp[:, j, :, e]
+            acc = (acc + (v * v).astype(np.float32)).astype(np.float32)
+    for o in (16, 8, 4, 2, 1):
+        acc = (acc + acc[:, np.arange(32) ^ o]).astype(np.float32)
+    total = acc[:, 0]
+    ms = (total / F(N)).astype(np.float32)
+    with np.errstate(divide="ignore", invalid="ignore", over="ignore"):       # an all-zero row with eps = 0 is 0 / 0 = NaN, by definition
+        r = (F(1.0) / np.sqrt((ms + F(eps)).astype(np.float32)).astype(np.float32)).astype(np.float32)
+        y = ((x * r[:, None]).astype(np.float32) * w[None, :]).astype(np.float32)
+    return f32_to_bf16(y)
+
+
+def add_bf16(a_bits, b_bits):
+    """Residual addition: bf16(a + b), one fp32 addition."""
+    return f32_to_bf16((bf16_to_f32(a_bits) + bf16_to_f32(b_bits)).astype(np.float32))

@@ -27,7 +27,8 @@ EXPORTED = [
     "rudder_linear_static_max_workspace_bytes", "rudder_linear_static",
     "rudder_block_profile", "rudder_block_host_staging_bytes", "rudder_block_host",
     "rudder_quantize_activations", "rudder_linear_dump_acc", "rudder_device_status", "rudder_status_string",
-    "rudder_gelu", "rudder_selftest_wait_timeout",
+    "rudder_gelu", "rudder_selftest_wait_timeout", "rudder_rmsnorm", "rudder_add",
+    "rudder_block_dit", "rudder_block_dit_workspace_bytes",
 ]
 
 
@@ -45,6 +46,11 @@ class _ScaleTable(ctypes.Structure):
 class _Segments(ctypes.Structure):
     _fields_ = [("seg_offsets", ctypes.POINTER(ctypes.c_int32)), ("seg_stream", ctypes.POINTER(ctypes.c_int32)),
                 ("n_seg", ctypes.c_int)]
+
+
+class _BlockGlue(ctypes.Structure):
+    _fields_ = [("norm1_weight", ctypes.c_void_p), ("norm2_weight", ctypes.c_void_p), ("eps", ctypes.c_float),
+                ("out", ctypes.c_void_p), ("ldout", ctypes.c_int64)]
 
 
 class _BlockArgs(ctypes.Structure):
@@ -97,6 +103,11 @@ def lib() -> ctypes.CDLL:
         L.rudder_device_status.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32)]
         L.rudder_gelu.argtypes = [vp, i64, i32, i32, vp, i64, vp]
         L.rudder_selftest_wait_timeout.argtypes = [ctypes.c_longlong, vp]
+        L.rudder_rmsnorm.argtypes = [vp, i64, i32, i32, vp, ctypes.c_float, vp, i64, vp]
+        L.rudder_add.argtypes = [vp, i64, vp, i64, i32, i32, vp, i64, vp]
+        L.rudder_block_dit_workspace_bytes.restype = sz
+        L.rudder_block_dit_workspace_bytes.argtypes = [ctypes.POINTER(_BlockArgs), i32]
+        L.rudder_block_dit.argtypes = [ctypes.POINTER(_BlockArgs), ctypes.POINTER(_BlockGlue), i32, ctypes.POINTER(_Segments), i32, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -351,3 +362,39 @@ def rudder_device_status():
 def rudder_selftest_wait_timeout(limit_cycles: int = 1_000_000, stream=None):
     """One warp waits `limit_cycles` SM clocks on a barrier nobody signals, gives up and records the time-out."""
     _check(lib().rudder_selftest_wait_timeout(int(limit_cycles), _stream(stream)), "rudder_selftest_wait_timeout")
+
+
+def rudder_rmsnorm(X: torch.Tensor, weight: torch.Tensor, eps: float, Y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Y = bf16((x / sqrt(mean(x^2) + eps)) * weight) per row, in the bit-defined form of the DiT block glue."""
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    assert weight.is_cuda and weight.dtype == torch.float32 and weight.is_contiguous() and weight.numel() == X.shape[1]
+    M, N = X.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    _check(lib().rudder_rmsnorm(_ptr(X), X.stride(0), int(M), int(N), _ptr(weight), ctypes.c_float(eps), _ptr(Y), Y.stride(0),
+                                _stream(stream)), "rudder_rmsnorm")
+    return Y
+
+
+def rudder_add(A: torch.Tensor, B: torch.Tensor, Y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Y = bf16(A + B), elementwise (the residual addition of the DiT block glue)."""
+    assert A.is_cuda and B.is_cuda and A.dtype == B.dtype == torch.bfloat16 and A.shape == B.shape and A.stride(1) == B.stride(1) == 1
+    M, N = A.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
+    _check(lib().rudder_add(_ptr(A), A.stride(0), _ptr(B), B.stride(0), int(M), int(N), _ptr(Y), Y.stride(0), _stream(stream)), "rudder_add")
+    return Y
+
+
+def rudder_block_dit_workspace_bytes(args: BlockArgs, M: int) -> int:
+    return int(lib().rudder_block_dit_workspace_bytes(ctypes.byref(args.c), int(M)))
+
+
+def rudder_block_dit(args: BlockArgs, norm1_weight: torch.Tensor, norm2_weight: torch.Tensor, eps: float, out: torch.Tensor, M: int,
+                     seg: Segments, step: int, workspace: torch.Tensor, stream=None):
+    """One DiT block end to end from args.x[0]: norm -> QKV -> O (V third) -> + x -> norm -> up -> GELU -> down -> + h."""
+    glue = _BlockGlue(norm1_weight.data_ptr(), norm2_weight.data_ptr(), float(eps), out.data_ptr(), out.stride(0))
+    wp, wb = _aligned(workspace)
+    _check(lib().rudder_block_dit(ctypes.byref(args.c), ctypes.byref(glue), int(M), ctypes.byref(seg.c), int(step), wp, wb,
+                                  _stream(stream)), "rudder_block_dit")
+    return out

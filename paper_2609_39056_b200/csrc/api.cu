@@ -496,6 +496,71 @@ size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M)
     return total;
 }
 
+// Workspace of rudder_block_dit: the four linears, the staged GELU output (M x F) and three M x H buffers
+// (normalised input of the attention half, the first residual sum, normalised input of the MLP half).
+static size_t dit_workspace_bytes(const rudder_block_args* args, int M)
+{
+    if (!args || M < 1) return 0;
+    size_t total = 0;
+    for (int l = 0; l < 4; ++l) {
+        if (!args->w[l]) return 0;
+        total += workspace_bytes_for(args->w[l], M);
+    }
+    total += align_up(static_cast<size_t>(M) * args->w[3]->K * 2, 256);
+    total += 3 * align_up(static_cast<size_t>(M) * args->w[0]->K * 2, 256);
+    return total;
+}
+
+static rudder_status block_dit_impl(const rudder_block_args* args, const rudder_block_glue* glue, int M, const rudder_segments* seg,
+                                    int step, void* workspace, size_t workspace_bytes, cudaStream_t st)
+{
+    if (!args || !glue || !glue->norm1_weight || !glue->norm2_weight || !glue->out) return RUDDER_ERR_ARG;
+    for (int l = 0; l < 4; ++l)
+        if (!args->w[l] || !args->tab[l] || !args->y[l] || !on_weights_device(args->w[l])) return RUDDER_ERR_ARG;
+    if (!args->x[0] || args->x[1] || args->x[2] || args->x[3]) return RUDDER_ERR_ARG;      // the block runs from x[0] alone
+    const int H = args->w[0]->K, F = args->w[2]->N;
+    if (args->w[0]->N != 3 * H || args->w[1]->K != H || args->w[1]->N != H || args->w[2]->K != H || args->w[3]->K != F || args->w[3]->N != H)
+        return RUDDER_ERR_SHAPE;
+    if (!(glue->eps >= 0.0f)) return RUDDER_ERR_ARG;
+    const size_t need = dit_workspace_bytes(args, M);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < need || need == 0) return RUDDER_ERR_WORKSPACE;
+    if (!aligned(args->x[0], 16) || args->ldx[0] % 8 != 0 || args->ldx[0] < H || !aligned(glue->out, 16) || glue->ldout % 8 != 0 || glue->ldout < H ||
+        !aligned(glue->norm1_weight, 16) || !aligned(glue->norm2_weight, 16))
+        return RUDDER_ERR_ALIGN;
+    for (int l = 0; l < 4; ++l) {
+        SegParams sp;
+        rudder_status s = check_table_and_segments(seg, step, args->tab[l], M, &sp);
+        if (s != RUDDER_OK) return s;
+        if (!aligned(args->y[l], 16) || args->ldy[l] % 8 != 0 || args->ldy[l] < args->w[l]->N) return RUDDER_ERR_ALIGN;
+    }
+    rudder_status s = ensure_init();
+    if (s != RUDDER_OK) return s;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    size_t lin_off[4], off = 0;
+    for (int l = 0; l < 4; ++l) { lin_off[l] = off; off += workspace_bytes_for(args->w[l], M); }
+    uint16_t* gelu_buf = reinterpret_cast<uint16_t*>(ws + off); off += align_up(static_cast<size_t>(M) * F * 2, 256);
+    uint16_t* n1 = reinterpret_cast<uint16_t*>(ws + off);       off += align_up(static_cast<size_t>(M) * H * 2, 256);
+    uint16_t* h1 = reinterpret_cast<uint16_t*>(ws + off);       off += align_up(static_cast<size_t>(M) * H * 2, 256);
+    uint16_t* n2 = reinterpret_cast<uint16_t*>(ws + off);
+    const int sms = sm_count();
+    auto lin = [&](int l, const uint16_t* x, int64_t ldx) {
+        return linear_impl(args->w[l], x, ldx, M, seg, step, args->tab[l], args->bias[l], args->y[l], args->ldy[l], ws + lin_off[l],
+                           workspace_bytes_for(args->w[l], M), st, nullptr, 0, 0, 0, 0, nullptr);
+    };
+    // attention half: h = x + O(V(QKV(norm1(x))))   (the V third of the QKV output stands in for attention, which stays outside)
+    if (launch_rmsnorm(args->x[0], args->ldx[0], glue->norm1_weight, glue->eps, n1, H, M, H, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if ((s = lin(0, n1, H)) != RUDDER_OK) return s;
+    if ((s = lin(1, args->y[0] + 2 * static_cast<size_t>(H), args->ldy[0])) != RUDDER_OK) return s;
+    if (launch_add(args->x[0], args->ldx[0], args->y[1], args->ldy[1], h1, H, M, H, sms, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    // MLP half: out = h + down(gelu(up(norm2(h))))
+    if (launch_rmsnorm(h1, H, glue->norm2_weight, glue->eps, n2, H, M, H, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if ((s = lin(2, n2, H)) != RUDDER_OK) return s;
+    if (launch_gelu(args->y[2], args->ldy[2], gelu_buf, F, M, F, sms, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if ((s = lin(3, gelu_buf, F)) != RUDDER_OK) return s;
+    if (launch_add(h1, H, args->y[3], args->ldy[3], glue->out, glue->ldout, M, H, sms, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    return RUDDER_OK;
+}
+
 static rudder_status block_impl(const rudder_block_args* args, int M, const rudder_segments* seg, int step, void* workspace,
                                 size_t workspace_bytes, void* stream, cudaEvent_t* ev /* [9] or nullptr */)
 {
@@ -556,6 +621,14 @@ rudder_status rudder_block(const rudder_block_args* args, int M, const rudder_se
                            size_t workspace_bytes, void* stream)
 {
     return block_impl(args, M, seg, step, workspace, workspace_bytes, stream, nullptr);
+}
+
+size_t rudder_block_dit_workspace_bytes(const rudder_block_args* args, int M) { return dit_workspace_bytes(args, M); }
+
+rudder_status rudder_block_dit(const rudder_block_args* args, const rudder_block_glue* glue, int M, const rudder_segments* seg, int step,
+                               void* workspace, size_t workspace_bytes, void* stream)
+{
+    return block_dit_impl(args, glue, M, seg, step, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
 }
 
 rudder_status rudder_block_profile(const rudder_block_args* args, int M, const rudder_segments* seg, int step,
@@ -723,6 +796,23 @@ rudder_status rudder_gelu(const uint16_t* X, int64_t ldx, int M, int N, uint16_t
     rudder_status s = ensure_init();
     if (s != RUDDER_OK) return s;
     return launch_gelu(X, ldx, Y, ldy, M, N, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? RUDDER_OK : RUDDER_ERR_CUDA;
+}
+
+rudder_status rudder_rmsnorm(const uint16_t* X, int64_t ldx, int M, int N, const float* weight, float eps, uint16_t* Y, int64_t ldy, void* stream)
+{
+    if (!X || !Y || !weight || !(eps >= 0.0f)) return RUDDER_ERR_ARG;
+    if (M < 1 || N < 8 || N % 8 != 0) return RUDDER_ERR_SHAPE;
+    if (!aligned(X, 16) || !aligned(Y, 16) || !aligned(weight, 16) || ldx % 8 != 0 || ldy % 8 != 0 || ldx < N || ldy < N) return RUDDER_ERR_ALIGN;
+    return launch_rmsnorm(X, ldx, weight, eps, Y, ldy, M, N, static_cast<cudaStream_t>(stream)) == cudaSuccess ? RUDDER_OK : RUDDER_ERR_CUDA;
+}
+
+rudder_status rudder_add(const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, int M, int N, uint16_t* Y, int64_t ldy, void* stream)
+{
+    if (!A || !B || !Y) return RUDDER_ERR_ARG;
+    if (M < 1 || N < 8 || N % 8 != 0) return RUDDER_ERR_SHAPE;
+    if (!aligned(A, 16) || !aligned(B, 16) || !aligned(Y, 16) || lda % 8 != 0 || ldb % 8 != 0 || ldy % 8 != 0 || lda < N || ldb < N || ldy < N)
+        return RUDDER_ERR_ALIGN;
+    return launch_add(A, lda, B, ldb, Y, ldy, M, N, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? RUDDER_OK : RUDDER_ERR_CUDA;
 }
 
 rudder_status rudder_selftest_wait_timeout(long long limit_cycles, void* stream)

@@ -1,6 +1,6 @@
 // BF16 glue between the quantized linears of a chained DiT block (the paper keeps GELU in BF16,
-// outside the quantized path: Appendix "Quantization").  Only what a chain of rudder_linear calls
-// needs to run back to back on the device: an elementwise GELU.
+// outside the quantized path, like normalisation and residual additions: Appendix "Quantization").  What a
+// chain of rudder_linear calls needs to run back to back on the device: GELU, RMS normalisation, residual add.
 //
 // GELU is taken in its tanh form, g(x) = x/2 (1 + tanh(sqrt(2/pi) (x + 0.044715 x^3))), with tanh
 // replaced by its [7/6] Pade approximant
@@ -64,7 +64,97 @@ __global__ void __launch_bounds__(256) gelu_bf16_kernel(const uint16_t* __restri
     }
 }
 
+// RMS normalisation of the rows of X with a weight per channel: y = bf16(((x * r) * w)), r = 1 / sqrt(mean(x^2) + eps).
+// (The paper keeps normalisation in BF16 and does not say which; reading: RMSNorm with a learned weight.)
+// Bit-defined like the GELU: one warp per row; lane l takes the 8-value pieces l, l + 32, ... in order and adds
+// x * x (product and sum rounded separately) into one fp32 partial; the 32 partials are combined by the
+// butterfly l ^ 16, 8, 4, 2, 1 (every lane ends with the same bits); mean = sum / N, r = 1 / sqrt(mean + eps) with
+// IEEE division and square root.
+__global__ void __launch_bounds__(256) rmsnorm_bf16_kernel(const uint16_t* __restrict__ X, int64_t ldx, const float* __restrict__ w,
+                                                           float eps, uint16_t* __restrict__ Y, int64_t ldy, int M, int N)
+{
+    const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    const int chunks = N >> 3;
+    const uint4* xr = reinterpret_cast<const uint4*>(X + static_cast<size_t>(row) * ldx);
+    float s = 0.0f;
+    for (int c = lane; c < chunks; c += 32) {
+        const uint4 v = xr[c];
+        const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(wds[i] << 16), hi = __uint_as_float(wds[i] & 0xFFFF0000u);
+            s = __fadd_rn(s, __fmul_rn(lo, lo));
+            s = __fadd_rn(s, __fmul_rn(hi, hi));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
+    const float r = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(s, static_cast<float>(N)), eps)));
+    uint4* yr = reinterpret_cast<uint4*>(Y + static_cast<size_t>(row) * ldy);
+    for (int c = lane; c < chunks; c += 32) {
+        const uint4 v = xr[c];
+        const float4 w0 = __ldg(reinterpret_cast<const float4*>(w) + 2 * c), w1 = __ldg(reinterpret_cast<const float4*>(w) + 2 * c + 1);
+        const float ww[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
+        const uint32_t wds[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(wds[i] << 16), hi = __uint_as_float(wds[i] & 0xFFFF0000u);
+            const float a = __fmul_rn(__fmul_rn(lo, r), ww[2 * i]), b = __fmul_rn(__fmul_rn(hi, r), ww[2 * i + 1]);
+            o[i] = static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(a))) |
+                   (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(b))) << 16);
+        }
+        yr[c] = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+// Residual addition, elementwise: y = bf16(a + b), one fp32 addition.
+__global__ void __launch_bounds__(256) add_bf16_kernel(const uint16_t* __restrict__ A, int64_t lda, const uint16_t* __restrict__ B, int64_t ldb,
+                                                       uint16_t* __restrict__ Y, int64_t ldy, int M, int N)
+{
+    const int chunks = N >> 3;
+    const long long total = static_cast<long long>(M) * chunks;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int row = static_cast<int>(i / chunks);
+        const int c = static_cast<int>(i - static_cast<long long>(row) * chunks);
+        const uint4 a = *reinterpret_cast<const uint4*>(A + static_cast<size_t>(row) * lda + 8 * c);
+        const uint4 b = *reinterpret_cast<const uint4*>(B + static_cast<size_t>(row) * ldb + 8 * c);
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float lo = __fadd_rn(__uint_as_float(aw[j] << 16), __uint_as_float(bw[j] << 16));
+            const float hi = __fadd_rn(__uint_as_float(aw[j] & 0xFFFF0000u), __uint_as_float(bw[j] & 0xFFFF0000u));
+            o[j] = static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(lo))) |
+                   (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(hi))) << 16);
+        }
+        *reinterpret_cast<uint4*>(Y + static_cast<size_t>(row) * ldy + 8 * c) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_rmsnorm(const uint16_t* X, int64_t ldx, const float* w, float eps, uint16_t* Y, int64_t ldy, int M, int N, cudaStream_t st)
+{
+    const int blocks = (M * 32 + 255) / 256;
+    rmsnorm_bf16_kernel<<<blocks, 256, 0, st>>>(X, ldx, w, eps, Y, ldy, M, N);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_add(const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, uint16_t* Y, int64_t ldy, int M, int N, int sm_count,
+                       cudaStream_t st)
+{
+    const long long total = static_cast<long long>(M) * (N >> 3);
+    long long blocks = (total + 255) / 256;
+    const long long cap = static_cast<long long>(sm_count > 0 ? sm_count : 148) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    add_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, st>>>(A, lda, B, ldb, Y, ldy, M, N);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_gelu(const uint16_t* X, int64_t ldx, uint16_t* Y, int64_t ldy, int M, int N, int sm_count, cudaStream_t st)
 {

@@ -101,3 +101,21 @@ def test_config4_small_m(rd, scheme, M, KN):
         check_output(bf16_to_np(Y), out["y64"])
     last, where = rd.rudder_device_status()
     assert last == 0, (last, where)
+
+
+@pytest.mark.parametrize("scheme,group", [("w4a8", 64), ("w4a8", 0), ("w4a4", 64), ("nvfp4", 16)])
+def test_cross_attention_kv_projections(rd, scheme, group):
+    """The cross-attention key and value projections: one global-text region each (a single segment of one
+    stream), 512 x 1024 -> 2048, every row against the oracle at three steps."""
+    cfg = wl.config(5, scheme)
+    for inp in cfg.draw():
+        G = group or inp.K
+        g = GpuLinear(rd, inp, scheme, G)
+        ref_w = oracle_pack(inp, scheme, G)
+        assert len(inp.seg_stream) == 1 and inp.S == 1
+        rows = np.arange(inp.M, dtype=np.int32)
+        for step in (0, 5, 9):
+            Y = rd.rudder_linear(g.w, g.X, g.seg, step, g.tab, g.bias)
+            check_linear_rows(rd, g, inp, ref_w, scheme, Y, step, rows)
+    last, where = rd.rudder_device_status()
+    assert last == 0, (last, where)

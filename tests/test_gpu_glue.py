@@ -80,3 +80,75 @@ def test_chained_block(rd, scheme, G):
         rd.rudder_block(bad, M, seg, step, ws)
     last, where = rd.rudder_device_status()
     assert last == 0, (last, where)
+
+
+@pytest.mark.parametrize("M,N", [(1, 8), (37, 264), (70, 2048), (5, 3072), (130, 12288)])
+def test_rmsnorm_and_add_bit_exact(rd, M, N):
+    rng = np.random.default_rng(900 + N)
+    xb = glue.f32_to_bf16((rng.standard_normal((M, N)) * 3.0).astype(np.float32))
+    yb = glue.f32_to_bf16((rng.standard_normal((M, N)) * 0.7).astype(np.float32))
+    if M > 2:
+        xb[1] = 0                                                  # an all-zero row
+    w = (1.0 + 0.1 * rng.standard_normal(N)).astype(np.float32)
+    X, Y2, W = to_dev_bf16(xb), to_dev_bf16(yb), torch.from_numpy(w).cuda()
+    for eps in (1e-6, 0.0) if M > 2 else (1e-6,):
+        got = bf16_to_np(rd.rudder_rmsnorm(X, W, eps))
+        want = glue.rmsnorm_bf16(xb, w, eps)
+        if eps == 0.0 and M > 2:                                   # 0 / 0 row: NaN on both sides
+            assert np.isnan(glue.bf16_to_f32(got[1])).all() and np.isnan(glue.bf16_to_f32(want[1])).all()
+            got, want = np.delete(got, 1, 0), np.delete(want, 1, 0)
+        assert np.array_equal(got, want)
+    assert np.array_equal(bf16_to_np(rd.rudder_add(X, Y2)), glue.add_bf16(xb, yb))
+    # strided views
+    wide = torch.zeros((M, N + 16), dtype=torch.bfloat16, device="cuda")
+    wide[:, 8:N + 8] = X
+    out = torch.full((M, N + 8), 5.0, dtype=torch.bfloat16, device="cuda")
+    rd.rudder_rmsnorm(wide[:, 8:N + 8], W, 1e-6, Y=out[:, :N])
+    assert np.array_equal(bf16_to_np(out[:, :N].contiguous()), glue.rmsnorm_bf16(xb, w, 1e-6)) and (out[:, N:] == 5.0).all().item()
+
+
+@pytest.mark.parametrize("scheme,G", [("w4a8", 64), ("w4a8", 256), ("nvfp4", 16)])
+def test_dit_block_with_bf16_glue(rd, scheme, G):
+    """rudder_block_dit: every glue step is the oracle's bit for bit, every linear is within tolerance of the
+    oracle fed the very input the GPU gave it."""
+    H, F, M = 256, 1024, 70
+    shapes = [(H, 3 * H), (H, H), (H, F), (F, H)]
+    layers = [GpuLinear(rd, wl.tiny(seed=800 + i, M=M, K=K, N=N, T=2), scheme, G if G != 256 else K) for i, (K, N) in enumerate(shapes)]
+    seg, step = layers[0].seg, 1
+    rng = np.random.default_rng(77)
+    w1 = (1.0 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    w2 = (1.0 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    W1, W2 = torch.from_numpy(w1).cuda(), torch.from_numpy(w2).cuda()
+    eps = 1e-6
+    ys = [torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda") for _, N in shapes]
+    out = torch.full((M, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    bargs = rd.BlockArgs([l.w for l in layers], [l.tab for l in layers], [l.bias for l in layers], [layers[0].X, None, None, None], ys)
+    ws = torch.empty(rd.rudder_block_dit_workspace_bytes(bargs, M) + 256, dtype=torch.uint8, device="cuda")
+    rd.rudder_block_dit(bargs, W1, W2, eps, out, M, seg, step, ws)
+    torch.cuda.synchronize()
+    x0 = bf16_to_np(layers[0].X)
+    y = [bf16_to_np(t) for t in ys]
+    # the glue, recomputed by the oracle from the GPU's own linear outputs
+    n1 = glue.rmsnorm_bf16(x0, w1, eps)
+    h1 = glue.add_bf16(x0, y[1])
+    n2 = glue.rmsnorm_bf16(h1, w2, eps)
+    ge = glue.gelu_bf16(y[2])
+    assert np.array_equal(bf16_to_np(out), glue.add_bf16(h1, y[3]))
+    ins = [n1, np.ascontiguousarray(y[0][:, 2 * H:3 * H]), n2, ge]
+    for l, g in enumerate(layers):
+        ref_w = oracle_pack(g.inp, scheme, g.group)
+        o = oracle.rudder_linear(ins[l], ref_w, g.inp.gamma, None, step, 0, layers[0].inp.seg_offsets, layers[0].inp.seg_stream,
+                                 scheme, g.inp.bias)
+        check_output(y[l], o["y64"], **({"rel": 2e-2} if scheme == "nvfp4" else {}))
+        # and the same layer through rudder_linear on the oracle's glue output gives the block's bits: the block
+        # really fed that input
+        assert torch.equal(ys[l], rd.rudder_linear(g.w, to_dev_bf16(ins[l]), seg, step, g.tab, g.bias)), f"layer {l}"
+    # replay inputs are refused (the block runs from x[0] alone), and so are shapes that do not form a block
+    bad = rd.BlockArgs([l.w for l in layers], [l.tab for l in layers], [l.bias for l in layers], [layers[0].X, layers[1].X, None, None], ys)
+    with pytest.raises(rd.RudderError):
+        rd.rudder_block_dit(bad, W1, W2, eps, out, M, seg, step, ws)
+    bad2 = rd.BlockArgs([layers[0].w, layers[2].w, layers[2].w, layers[3].w], [l.tab for l in layers], [None] * 4, [layers[0].X, None, None, None], ys)
+    with pytest.raises(rd.RudderError):
+        rd.rudder_block_dit(bad2, W1, W2, eps, out, M, seg, step, ws)
+    last, where = rd.rudder_device_status()
+    assert last == 0, (last, where)

@@ -115,7 +115,7 @@ def _block(H, F):
 
 
 def config(index: int, scheme: str | None = None, M: int | None = None, KN: int | None = None) -> Config:
-    """The five benchmark configurations.  ``scheme`` selects the variant where a configuration
+    """The five benchmark configurations, and (5) the cross-attention key / value workload.  ``scheme`` selects the variant where a configuration
     names several; ``M`` / ``KN`` select the point of the small-M sweep (configuration 4)."""
     if index == 0:
         return Config("cfg0_w4a8_linear_256x1024x1024", 0, scheme or "w4a8", 64, 1, 3,
@@ -136,6 +136,13 @@ def config(index: int, scheme: str | None = None, M: int | None = None, KN: int 
         sch = scheme or "w4a8"
         return Config(f"cfg4_{sch}_smallM_m{m}_kn{kn}", 4, sch, 64, 20, 3,
                       [(m // 4, PROPRIO), (m - m // 4, ACTION)], [("linear", kn, kn)], 0.01, 30.0)
+    if index == 5:
+        # Cross-attention key / value projections: the text conditioning forms ONE global region per projection
+        # (a single segment, a single stream), with its own per-step tables.  The paper gives neither the text
+        # length nor the widths: 512 text tokens of width 1024 projected to the block width of configuration 2.
+        sch = scheme or "w4a8"
+        return Config(f"cfg5_{sch}_crossattn_kv_m512_k1024_n2048", 5, sch, 64, 10, 1,
+                      [(M or 512, VIDEO)], [("k_proj", 1024, 2048), ("v_proj", 1024, 2048)], 0.01, 30.0)
     raise ValueError(index)
 
 
