@@ -9,7 +9,7 @@ action) tokens, 10 steps of tables).  The W4A8 block (configuration 2), the W4A4
 (configuration 3) and the small-M sweep (configuration 4) are measured in the same run and reported
 under "also" (rank 0, N = 1).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg2_g128|cfg2_perchannel|cfg2_perchannel_static|cfg2_chained|cfg3|cfg3_perchannel|cfg3_nvfp4|cfg4] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg2_g128|cfg2_perchannel|cfg2_perchannel_static|cfg2_chained|cfg2_perchannel_static_chained|cfg3|cfg3_perchannel|cfg3_nvfp4|cfg4] [--impl reference]
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded row sample.
 """
@@ -64,6 +64,10 @@ def workload_config(name: str):
         import dataclasses
         c = wl.config(2)
         return dataclasses.replace(c, name=c.name + "_chained")
+    if name == "cfg2_perchannel_static_chained":      # the same chain in the paper's setting: per-channel W4, one static threshold per step;
+        import dataclasses                            # the GELU then runs inside the down projection's prologue
+        c = wl.config(2)
+        return dataclasses.replace(c, name=c.name + "_per_channel_static_chained", group=0)
     if name == "cfg3_perchannel":                     # configuration 3 (W4A4-INT) with one scale per output channel
         import dataclasses
         c = wl.config(3, "w4a4")
@@ -151,7 +155,7 @@ def build_block(rd, cfg, torch, dev):
         ws.append(rd.rudder_pack_weights(W, d, scheme, cfg.group or l.K))     # group 0: one scale per output channel (G = K)
         del W, d
         gamma = torch.from_numpy(l.gamma).to(dev)
-        if cfg.name.endswith("_static"):
+        if cfg.name.endswith("_static") or cfg.name.endswith("_static_chained"):
             # input recipe, step 8: clip[t] = 99.9th percentile of |(x dinv) gamma[t, s(i)]| over all rows
             x = torch.from_numpy(l.X_bf16.view(np.int16)).to(dev).view(torch.bfloat16).float()
             x *= rd.rudder_weight_export(ws[-1])["dinv"][None, :]
@@ -544,7 +548,7 @@ def run_ours(args):
         del m, ws, tabs, biases, xs, ys, workspace, lins
         torch.cuda.empty_cache()
         also = {}
-        for name in ("cfg2", "cfg2_g128", "cfg2_perchannel", "cfg2_perchannel_static", "cfg2_chained", "cfg3", "cfg3_perchannel",
+        for name in ("cfg2", "cfg2_g128", "cfg2_perchannel", "cfg2_perchannel_static", "cfg2_chained", "cfg2_perchannel_static_chained", "cfg3", "cfg3_perchannel",
                      "cfg3_nvfp4"):
             if name == args.workload:
                 continue
@@ -574,7 +578,7 @@ def run_ours(args):
                                                               "nvfp4": "e2m1 x e2m1 (ue4m3 block scales) -> fp32"}[cfg.scheme],
             "data": "synthetic", "gpu_launches": 8 * args.steps,
             "config": {"workload": cfg.name, "scheme": cfg.scheme, "group": 16 if cfg.scheme == "nvfp4" else cfg.group, "M": M,
-                       "linears": {n: [K, N] for n, K, N in cfg.linears}, "range_mode": "static" if cfg.name.endswith("_static") else "per_token",
+                       "linears": {n: [K, N] for n, K, N in cfg.linears}, "range_mode": "static" if "_static" in cfg.name else "per_token",
                        "steps_of_tables": T, "tops_per_step": ops / 1e12,
                        "l2": f"working set per step {sum(alg_bytes) / 1e6:.0f} MB (inputs {sum(2 * M * K for _, K, _ in cfg.linears) / 1e6:.0f} MB) exceeds the 126 MB L2; no explicit flush",
                        "parallelism": f"replicas x{world} (rows independent, no collective)"},
@@ -630,7 +634,7 @@ def cpu_baseline(cfg, lins, target_s=15.0, impl_reference=False):
     for l in lins:
         packs.append(oracle.pack_nvfp4(l.W, l.d) if cfg.scheme == "nvfp4" else oracle.pack_int4(l.W, l.d, cfg.group or l.K))
     M = cfg.M
-    static = cfg.name.endswith("_static")
+    static = "_static" in cfg.name
     clips = []
     for l, pw in zip(lins, packs):
         if not static:

@@ -176,6 +176,10 @@ typedef struct {
  *                 stays outside this library; requires N_0 == 3 K_1;
  *   up   (l = 2): the O output as it is (no norm / residual); requires N_1 == K_2;
  *   down (l = 3): rudder_gelu of the up output, staged at the end of the workspace; requires N_2 == K_3.
+ *                 When the down projection's table has a static range (RUDDER_RANGE_STATIC: the paper's calibrated
+ *                 threshold, Section 4.3) and an integer scheme, the GELU is applied INSIDE its prologue: with a_i = c_tau
+ *                 the requantisation needs no row reduction, so one elementwise pass reads the up output, applies
+ *                 the GELU and writes Q_X and r directly; the activated tensor is never stored (same bits either way).
  * A shape that does not chain returns RUDDER_ERR_SHAPE.  rudder_block_workspace_bytes accounts for the
  * staged GELU output (M x K_3 bf16) when x[3] is NULL.  rudder_block_host takes no NULL inputs. */
 size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M);
@@ -231,6 +235,12 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
                                           const rudder_segments* seg, int step,
                                           const rudder_scale_table* tab, void* codes,
                                           uint8_t* block_scales, float* row_scale, void* stream);
+/* The fused pass of a chained down projection alone (see rudder_block): X is the tensor BEFORE the GELU; the codes
+ * (int8 [M, K], one per byte) and row scales are those of bf16(gelu(X)).  Static range and integer schemes only
+ * (RUDDER_ERR_UNSUPPORTED otherwise). */
+rudder_status rudder_gelu_quantize_activations(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M,
+                                               const rudder_segments* seg, int step, const rudder_scale_table* tab,
+                                               void* codes, float* row_scale, void* stream);
 /* rudder_linear that also writes the INT32 group accumulators C^(g) (Section 4.4: "accumulates
  * C = Q_X Q_W in INT32") of rows [row0, row0+rows) x columns [col0, col0+cols) into
  * acc int32 [K/group][rows][cols].  Integer schemes only.  row0 % 128 == 0 and col0 % 64 == 0. */

@@ -28,7 +28,7 @@ EXPORTED = [
     "rudder_block_profile", "rudder_block_host_staging_bytes", "rudder_block_host",
     "rudder_quantize_activations", "rudder_linear_dump_acc", "rudder_device_status", "rudder_status_string",
     "rudder_gelu", "rudder_selftest_wait_timeout", "rudder_rmsnorm", "rudder_add",
-    "rudder_block_dit", "rudder_block_dit_workspace_bytes",
+    "rudder_block_dit", "rudder_block_dit_workspace_bytes", "rudder_gelu_quantize_activations",
 ]
 
 
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.rudder_block_host.argtypes = [ctypes.POINTER(_BlockArgs), i32, ctypes.POINTER(_Segments), i32, vp, sz, vp, sz, vp]
         L.rudder_quantize_activations.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32,
                                                   ctypes.POINTER(_ScaleTable), vp, vp, vp, vp]
+        L.rudder_gelu_quantize_activations.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32,
+                                                       ctypes.POINTER(_ScaleTable), vp, vp, vp]
         L.rudder_linear_dump_acc.argtypes = [vp, vp, i64, i32, ctypes.POINTER(_Segments), i32,
                                              ctypes.POINTER(_ScaleTable), vp, vp, i64, vp, sz, vp,
                                              i32, i32, i32, i32, vp]
@@ -398,3 +400,14 @@ def rudder_block_dit(args: BlockArgs, norm1_weight: torch.Tensor, norm2_weight: 
     _check(lib().rudder_block_dit(ctypes.byref(args.c), ctypes.byref(glue), int(M), ctypes.byref(seg.c), int(step), wp, wb,
                                   _stream(stream)), "rudder_block_dit")
     return out
+
+
+def rudder_gelu_quantize_activations(w: Weight, X, seg, step, tab, stream=None):
+    """The fused GELU + static-range prologue of a chained layer alone -> (codes int8 [M, K], row_scale)."""
+    M = X.shape[0]
+    codes = torch.empty((M, w.K), dtype=torch.int8, device=X.device)
+    r = torch.empty(M, dtype=torch.float32, device=X.device)
+    _check(lib().rudder_gelu_quantize_activations(w.handle, _ptr(X), X.stride(0), M, ctypes.byref(seg.c), int(step),
+                                                  ctypes.byref(tab.c), _ptr(codes), _ptr(r), _stream(stream)),
+           "rudder_gelu_quantize_activations")
+    return codes, r

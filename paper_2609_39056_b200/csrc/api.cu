@@ -150,7 +150,8 @@ size_t workspace_bytes_for(const rudder_weight* w, int M)
 rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M, const rudder_segments* seg,
                           int step, const rudder_scale_table* tab, const float* bias, uint16_t* Y, int64_t ldy,
                           void* workspace, size_t workspace_bytes, cudaStream_t st, int32_t* acc, int row0, int rows,
-                          int col0, int cols, cudaEvent_t* ev = nullptr /* ev[1] recorded after the prologue, ev[2] after the GEMM */)
+                          int col0, int cols, cudaEvent_t* ev = nullptr /* ev[1] recorded after the prologue, ev[2] after the GEMM */,
+                          bool gelu_first = false /* X is the tensor before the GELU: the prologue applies it (static range only) */)
 {
     if (!w || !X || !Y) return RUDDER_ERR_ARG;
     if (!on_weights_device(w)) return RUDDER_ERR_ARG;
@@ -176,6 +177,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     a.clip_step = (tab->mode == RUDDER_RANGE_STATIC) ? tab->clip + step : nullptr;
     a.seg = sp;
 
+    if (gelu_first && (a.clip_step == nullptr || w->scheme == RUDDER_W4A4_NVFP4)) return RUDDER_ERR_UNSUPPORTED;
     if (w->scheme == RUDDER_W4A4_NVFP4) {
         uint8_t* ws = static_cast<uint8_t*>(workspace);
         uint8_t* codes4 = ws;
@@ -213,7 +215,8 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
     float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
     if (gemm_i8_fewrows_applies(M, w->N, w->K, w->G)) {
         // A handful of rows: the light prologue (int8 codes, whatever the weight layout) and the register-level GEMM.
-        if (launch_actq_int(a, qmax_of(w->scheme), false, codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if ((gelu_first ? launch_actq_gelu_static(a, qmax_of(w->scheme), false, codes, w->K, r, sm_count(), st)
+                        : launch_actq_int(a, qmax_of(w->scheme), false, codes, w->K, r, st)) != cudaSuccess) return RUDDER_ERR_CUDA;
         if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
         GemmI8FewRowsArgs f;
         f.codes = codes; f.ldc = w->K; f.row_scale = r; f.wq = w->codes; f.signmag = w->f8 != 0;
@@ -236,7 +239,8 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
         a.zero_ints = g.counters;
         a.n_zero = ((M + plan.token_tile - 1) / plan.token_tile) * ((w->N + 127) / 128);
     }
-    if (launch_actq_int(a, qmax_of(w->scheme), w->f8 != 0, codes, w->K, r, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+    if ((gelu_first ? launch_actq_gelu_static(a, qmax_of(w->scheme), w->f8 != 0, codes, w->K, r, sm_count(), st)
+                    : launch_actq_int(a, qmax_of(w->scheme), w->f8 != 0, codes, w->K, r, st)) != cudaSuccess) return RUDDER_ERR_CUDA;
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
 
     const int tt = plan.token_tile;
@@ -496,6 +500,12 @@ size_t rudder_block_workspace_bytes(const rudder_block_args* args, int M)
     return total;
 }
 
+// The GELU in front of a chained layer moves into that layer's prologue when the range is static and the codes are integers.
+static bool gelu_fuses(const rudder_weight* w, const rudder_scale_table* tab)
+{
+    return tab->mode == RUDDER_RANGE_STATIC && tab->clip != nullptr && w->scheme != RUDDER_W4A4_NVFP4;
+}
+
 // Workspace of rudder_block_dit: the four linears, the staged GELU output (M x F) and three M x H buffers
 // (normalised input of the attention half, the first residual sum, normalised input of the MLP half).
 static size_t dit_workspace_bytes(const rudder_block_args* args, int M)
@@ -555,8 +565,14 @@ static rudder_status block_dit_impl(const rudder_block_args* args, const rudder_
     // MLP half: out = h + down(gelu(up(norm2(h))))
     if (launch_rmsnorm(h1, H, glue->norm2_weight, glue->eps, n2, H, M, H, st) != cudaSuccess) return RUDDER_ERR_CUDA;
     if ((s = lin(2, n2, H)) != RUDDER_OK) return s;
-    if (launch_gelu(args->y[2], args->ldy[2], gelu_buf, F, M, F, sms, st) != cudaSuccess) return RUDDER_ERR_CUDA;
-    if ((s = lin(3, gelu_buf, F)) != RUDDER_OK) return s;
+    if (gelu_fuses(args->w[3], args->tab[3])) {
+        s = linear_impl(args->w[3], args->y[2], args->ldy[2], M, seg, step, args->tab[3], args->bias[3], args->y[3], args->ldy[3], ws + lin_off[3],
+                        workspace_bytes_for(args->w[3], M), st, nullptr, 0, 0, 0, 0, nullptr, true);
+        if (s != RUDDER_OK) return s;
+    } else {
+        if (launch_gelu(args->y[2], args->ldy[2], gelu_buf, F, M, F, sms, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if ((s = lin(3, gelu_buf, F)) != RUDDER_OK) return s;
+    }
     if (launch_add(h1, H, args->y[3], args->ldy[3], glue->out, glue->ldout, M, H, sms, st) != cudaSuccess) return RUDDER_ERR_CUDA;
     return RUDDER_OK;
 }
@@ -605,12 +621,16 @@ static rudder_status block_impl(const rudder_block_args* args, int M, const rudd
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     for (int l = 0; l < 4; ++l) {
         const size_t bytes = workspace_bytes_for(args->w[l], M);
-        if (l == 3 && args->x[3] == nullptr &&
+        // Chained down projection.  With a static range (the paper's calibrated threshold) its prologue has no row
+        // reduction, so the GELU is applied inside it, straight from the up output: no activated tensor is written
+        // or read back and the GELU launch goes away.  Otherwise GELU runs as a pass of its own into the staging buffer.
+        const bool fuse_gelu = l == 3 && args->x[3] == nullptr && gelu_fuses(args->w[3], args->tab[3]);
+        if (l == 3 && args->x[3] == nullptr && !fuse_gelu &&
             launch_gelu(args->y[2], args->ldy[2], gelu_buf, args->w[3]->K, M, args->w[3]->K, sm_count(), static_cast<cudaStream_t>(stream)) != cudaSuccess)
             return RUDDER_ERR_CUDA;
-        rudder_status s = linear_impl(args->w[l], x_eff[l], ldx_eff[l], M, seg, step, args->tab[l], args->bias[l],
-                                      args->y[l], args->ldy[l], ws, bytes, static_cast<cudaStream_t>(stream), nullptr, 0, 0,
-                                      0, 0, ev ? ev + 2 * l : nullptr);
+        rudder_status s = linear_impl(args->w[l], fuse_gelu ? args->y[2] : x_eff[l], fuse_gelu ? args->ldy[2] : ldx_eff[l], M, seg, step,
+                                      args->tab[l], args->bias[l], args->y[l], args->ldy[l], ws, bytes, static_cast<cudaStream_t>(stream),
+                                      nullptr, 0, 0, 0, 0, ev ? ev + 2 * l : nullptr, fuse_gelu);
         if (s != RUDDER_OK) return s;
         ws += bytes;
     }
@@ -782,6 +802,31 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
     // E4M3 bytes of the same integers, which are then decoded in place so that the caller sees integers.
     const bool e4m3 = w->f8 != 0 && !gemm_i8_fewrows_applies(M, w->N, w->K, w->G);     // the few-rows GEMM reads int8 whatever the weight layout
     if (launch_actq_int(a, qmax_of(w->scheme), e4m3, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
+    if (e4m3 && launch_e4m3_to_int8(static_cast<int8_t*>(codes), static_cast<size_t>(M) * w->K, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return RUDDER_ERR_CUDA;
+    return RUDDER_OK;
+}
+
+rudder_status rudder_gelu_quantize_activations(const rudder_weight* w, const uint16_t* X, int64_t ldx, int M, const rudder_segments* seg,
+                                               int step, const rudder_scale_table* tab, void* codes, float* row_scale, void* stream)
+{
+    if (!w || !X || !codes || !row_scale) return RUDDER_ERR_ARG;
+    if (!on_weights_device(w)) return RUDDER_ERR_ARG;
+    if (M < 1) return RUDDER_ERR_SHAPE;
+    SegParams sp;
+    rudder_status s = check_table_and_segments(seg, step, tab, M, &sp);
+    if (s != RUDDER_OK) return s;
+    if (!gelu_fuses(w, tab)) return RUDDER_ERR_UNSUPPORTED;
+    if (!aligned(X, 16) || ldx % 8 != 0 || ldx < w->K || !aligned(codes, 16)) return RUDDER_ERR_ALIGN;
+    ActqArgs a;
+    a.zero_ints = nullptr; a.n_zero = 0;
+    a.X = X; a.ldx = ldx; a.M = M; a.K = w->K; a.dinv = w->dinv;
+    a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
+    a.clip_step = tab->clip + step;
+    a.seg = sp;
+    const bool e4m3 = w->f8 != 0 && !gemm_i8_fewrows_applies(M, w->N, w->K, w->G);     // what production writes for this weight and shape
+    if (launch_actq_gelu_static(a, qmax_of(w->scheme), e4m3, static_cast<int8_t*>(codes), w->K, row_scale, sm_count(), static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     if (e4m3 && launch_e4m3_to_int8(static_cast<int8_t*>(codes), static_cast<size_t>(M) * w->K, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;

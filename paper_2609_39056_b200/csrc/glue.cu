@@ -135,7 +135,63 @@ __global__ void __launch_bounds__(256) add_bf16_kernel(const uint16_t* __restric
     }
 }
 
+// ---- GELU fused into the activation prologue of the layer behind it (static range) ----------------------
+// With the paper's static threshold c_tau (Section 4.3; Appendix "Quantization": one calibrated base scale
+// shared by all streams) the prologue of the down projection needs no row reduction: a_i = c_tau for every
+// row.  Requantising the up projection's output is then purely elementwise, so the GELU between the two
+// layers moves into the same pass: read the up output once, bf16(gelu(.)), v = (g * dinv_k) * gamma_s(i),
+// code = clip(round(v * q_max / c)), and r_i = (c / q_max) / gamma_s(i).  The activated tensor is never
+// written, the prologue never reads it back, and one launch goes away.  The arithmetic per element is
+// gelu_f32 above followed by scale8 / round8 of the prologue: the same bits as the two separate passes.
+__global__ void __launch_bounds__(256) actq_gelu_static_kernel(ActqArgs a, int qmax, int e4m3, int8_t* __restrict__ codes, int64_t ldc,
+                                                                float* __restrict__ r)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (blockIdx.x == 0 && a.zero_ints != nullptr)
+        for (int i = threadIdx.x; i < a.n_zero; i += blockDim.x) a.zero_ints[i] = 0;
+    const int chunks = a.K >> 3;
+    const long long total = static_cast<long long>(a.M) * chunks;
+    const float range = *a.clip_step;
+    const float qf = static_cast<float>(qmax);
+    const float inv = (range != 0.0f) ? __fdiv_rn(qf, range) : 0.0f;
+    const float4* dv = reinterpret_cast<const float4*>(a.dinv);
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int row = static_cast<int>(i / chunks);
+        const int c = static_cast<int>(i - static_cast<long long>(row) * chunks);
+        const float g = a.gamma_step[stream_of_row(a.seg, row)];
+        const uint4 x = *reinterpret_cast<const uint4*>(a.X + static_cast<size_t>(row) * a.ldx + 8 * c);
+        uint4 act;
+        act.x = gelu_pair(x.x); act.y = gelu_pair(x.y); act.z = gelu_pair(x.z); act.w = gelu_pair(x.w);
+        float v[8];
+        scale8(act, __ldg(dv + 2 * c), __ldg(dv + 2 * c + 1), g, v);
+        *reinterpret_cast<uint2*>(codes + static_cast<size_t>(row) * ldc + 8 * c) = e4m3 ? round8_e4m3(v, inv, qmax) : round8(v, inv, qmax);
+        if (c == 0) r[row] = (range != 0.0f) ? __fdiv_rn(__fdiv_rn(range, qf), g) : 0.0f;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_actq_gelu_static(const ActqArgs& a, int qmax, bool e4m3, int8_t* codes, int64_t ldc, float* r, int sm_count, cudaStream_t st)
+{
+    const long long total = static_cast<long long>(a.M) * (a.K >> 3);
+    long long blocks = (total + 255) / 256;
+    const long long cap = static_cast<long long>(sm_count > 0 ? sm_count : 148) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, actq_gelu_static_kernel, a, qmax, e4m3 ? 1 : 0, codes, ldc, r);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
 
 cudaError_t launch_rmsnorm(const uint16_t* X, int64_t ldx, const float* w, float eps, uint16_t* Y, int64_t ldy, int M, int N, cudaStream_t st)
 {

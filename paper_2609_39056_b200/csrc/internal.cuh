@@ -76,6 +76,8 @@ cudaError_t launch_import_nvfp4_scales(const uint8_t* sb_canonical, int N, int K
 cudaError_t launch_export_int4(const uint8_t* codes_il, int N, int K, uint8_t* canonical, bool signmag, cudaStream_t st);
 
 cudaError_t launch_gelu(const uint16_t* X, int64_t ldx, uint16_t* Y, int64_t ldy, int M, int N, int sm_count, cudaStream_t st);
+// GELU + static-range activation prologue in one elementwise pass (X is the tensor BEFORE the GELU; a.clip_step must be set)
+cudaError_t launch_actq_gelu_static(const ActqArgs& a, int qmax, bool e4m3, int8_t* codes, int64_t ldc, float* r, int sm_count, cudaStream_t st);
 cudaError_t launch_rmsnorm(const uint16_t* X, int64_t ldx, const float* w, float eps, uint16_t* Y, int64_t ldy, int M, int N, cudaStream_t st);
 cudaError_t launch_add(const uint16_t* A, int64_t lda, const uint16_t* B, int64_t ldb, uint16_t* Y, int64_t ldy, int M, int N, int sm_count,
                        cudaStream_t st);

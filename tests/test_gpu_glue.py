@@ -152,3 +152,47 @@ def test_dit_block_with_bf16_glue(rd, scheme, G):
         rd.rudder_block_dit(bad2, W1, W2, eps, out, M, seg, step, ws)
     last, where = rd.rudder_device_status()
     assert last == 0, (last, where)
+
+
+@pytest.mark.parametrize("scheme,G", [("w4a8", 0), ("w4a8", 64), ("w4a4", 64), ("w4a4", 0)])
+@pytest.mark.parametrize("M", [20, 300])
+def test_static_range_fuses_gelu_into_the_down_prologue(rd, scheme, G, M):
+    """Chained block whose down projection has the paper's static threshold: the GELU runs inside that layer's
+    prologue.  The codes and row scales of the fused pass are the oracle's (GELU, then static quantisation) bit
+    for bit, and the block's outputs are the bits of the unfused sequence."""
+    H, F = 256, 1024
+    shapes = [(H, 3 * H), (H, H), (H, F), (F, H)]
+    qmax = 127 if scheme == "w4a8" else 7
+    inps = [wl.tiny(seed=860 + i, M=M, K=K, N=N, T=2) for i, (K, N) in enumerate(shapes)]
+    step = 1
+    # thresholds: for the down projection a value that clips some of the activated values
+    clips = [np.array([3.0, 2.0], np.float32) for _ in shapes]
+    clips[3] = np.array([0.8, 0.35], np.float32)
+    layers = [GpuLinear(rd, inp, scheme, G or inp.K, 1, clips[i]) for i, inp in enumerate(inps)]
+    seg = layers[0].seg
+    ys = [torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda") for _, N in shapes]
+    bargs = rd.BlockArgs([l.w for l in layers], [l.tab for l in layers], [l.bias for l in layers], [layers[0].X, None, None, None], ys)
+    ws = torch.empty(rd.rudder_block_workspace_bytes(bargs, M) + 256, dtype=torch.uint8, device="cuda")
+    rd.rudder_block(bargs, M, seg, step, ws)
+    torch.cuda.synchronize()
+    # the fused pass alone against the oracle
+    y2 = bf16_to_np(ys[2])
+    codes, r = rd.rudder_gelu_quantize_activations(layers[3].w, ys[2], seg, step, layers[3].tab)
+    ref_w = oracle_pack(inps[3], scheme, G or inps[3].K)
+    rc, rr = oracle.quantize_int(glue.gelu_bf16(y2), ref_w["dinv"], inps[3].gamma, clips[3], step, 1, inps[0].seg_offsets,
+                                 inps[0].seg_stream, qmax)
+    assert np.array_equal(codes.cpu().numpy(), rc)
+    assert np.array_equal(r.cpu().numpy().view(np.uint32), rr.view(np.uint32))
+    assert (np.abs(rc) == qmax).any()                              # the threshold does clip
+    # the down output: the oracle on the GPU's own up output, and the unfused sequence bit for bit
+    _, y64 = oracle.linear_int(rc, rr, ref_w["qw"], ref_w["scales"], G or inps[3].K, inps[3].bias)
+    check_output(bf16_to_np(ys[3]), y64)
+    a2 = rd.rudder_gelu(ys[2])
+    assert torch.equal(ys[3], rd.rudder_linear(layers[3].w, a2, seg, step, layers[3].tab, layers[3].bias))
+    # per-token tables are not fused: the hook says so
+    pt = GpuLinear(rd, inps[3], scheme, G or inps[3].K)
+    with pytest.raises(rd.RudderError) as e:
+        rd.rudder_gelu_quantize_activations(pt.w, ys[2], seg, step, pt.tab)
+    assert e.value.status == rd.ERR_UNSUPPORTED
+    last, where = rd.rudder_device_status()
+    assert last == 0, (last, where)
