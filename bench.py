@@ -479,7 +479,8 @@ def run_ours(args):
         # the ncu summary of the small-M kernels is taken from.  Rank 0 only; the value is the sweep's
         # mean throughput.
         if rank == 0:
-            sweep = small_m_sweep(rd, torch, dev, pk, schemes=("w4a8",))
+            sweep = small_m_sweep(rd, torch, dev, pk, schemes=tuple(args.cfg4_schemes.split(",")), sizes=tuple(int(x) for x in args.cfg4_sizes.split(",")),
+                                  rows=tuple(int(x) for x in args.cfg4_rows.split(",")), cold=not args.no_cold)
             mean_us = float(np.mean([r["us_per_linear"] for r in sweep]))
             print(json.dumps({"metric": "small-M W4A8 linear (configuration 4), mean over M in {16,64,128,256}, K=N in {2048,4096}",
                               "value": float(np.mean([r["tops"] for r in sweep])), "unit": "TOPS", "n_gpus": 1,
@@ -703,6 +704,10 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     ap.add_argument("--no-bf16", action="store_true", help="skip the cuBLAS BF16 comparison")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--cfg4-schemes", default="w4a8", help="--workload cfg4: schemes of the sweep")
+    ap.add_argument("--cfg4-sizes", default="2048,4096", help="--workload cfg4: K = N values")
+    ap.add_argument("--cfg4-rows", default="16,64,128,256", help="--workload cfg4: M values")
+    ap.add_argument("--no-cold", action="store_true", help="--workload cfg4: skip the rotation over distinct weights")
     ap.add_argument("--sustain-seconds", type=float, default=2.0, help="length of the sustained leg of every block workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
