@@ -807,17 +807,24 @@ GemmI8Plan gemm_i8_plan(int M, int N, int K, int G, bool f8, bool dump)
         const bool shape_ok = G >= K || (G >= 128 && !f8);
         plan.persist = !dump && M > 256 && shape_ok && tiles >= static_cast<long long>(kPersistTilesPerSm) * sm_count;
     }
-    plan.token_tile = M > 256 ? 256 : (M > 32 ? 64 : 32);    // up to 256 tokens: small tiles, eight TMEM buffers
+    // Small tiles (eight TMEM buffers) and split K wherever 256-token tiles would leave more than half of
+    // the SMs without one: up to 256 rows always, above that while the 64-token tiles still fit one wave.
+    const int n_tiles = (N + BN - 1) / BN;
+    const long long tiles256 = static_cast<long long>((M + 255) / 256) * n_tiles;
+    const long long tiles64 = static_cast<long long>((M + 63) / 64) * n_tiles;
+    const bool small = M <= 256 || (tiles256 * 2 <= sm_count && tiles64 <= sm_count + sm_count / 12);
+    plan.token_tile = !small ? 256 : (M > 32 ? 64 : 32);
     plan.splitk = 1;
     plan.pdl = false;
-    if (dump || M > 256) return plan;
-    const int n_tiles = (N + BN - 1) / BN;
+    if (dump || !small) return plan;
     const int m_tiles = (M + plan.token_tile - 1) / plan.token_tile;
     const int base = m_tiles * n_tiles;
     const size_t m_pad = static_cast<size_t>(m_tiles) * plan.token_tile;
+    // Split K until about one CTA per SM, but leave every CTA at least four stages (deeper splits cost
+    // more in the reduction than they gain) and keep the fp32 partial sums within 4 MiB.
     int sk = 1;
-    while (sk < 16 && base * (sk * 2) <= sm_count + sm_count / 12 && (K / KSTAGE) % (sk * 2) == 0 && K / (sk * 2) >= 2 * KSTAGE &&
-           static_cast<size_t>(sk * 2) * N * m_pad * sizeof(float) <= (size_t(2) << 20))
+    while (sk < 16 && base * (sk * 2) <= sm_count + sm_count / 12 && (K / KSTAGE) % (sk * 2) == 0 && K / (sk * 2) >= 4 * KSTAGE &&
+           static_cast<size_t>(sk * 2) * N * m_pad * sizeof(float) <= (size_t(4) << 20))
         sk *= 2;
     plan.splitk = sk;
     plan.pdl = true;
