@@ -213,8 +213,8 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
 
     int8_t* codes = static_cast<int8_t*>(workspace);
     float* r = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up(static_cast<size_t>(M) * w->K, 256));
-    if (gemm_i8_fewrows_applies(M, w->N, w->K, w->G)) {
-        // A handful of rows: the light prologue (int8 codes, whatever the weight layout) and the register-level GEMM.
+    if (gemm_i8_register_path(M, w->N, w->K, w->G, w->f8 != 0)) {
+        // Up to a few hundred rows: the light prologue (int8 codes, whatever the weight layout) and a register-level GEMM.
         if ((gelu_first ? launch_actq_gelu_static(a, qmax_of(w->scheme), false, codes, w->K, r, sm_count(), st)
                         : launch_actq_int(a, qmax_of(w->scheme), false, codes, w->K, r, st)) != cudaSuccess) return RUDDER_ERR_CUDA;
         if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return RUDDER_ERR_CUDA;
@@ -223,7 +223,7 @@ rudder_status linear_impl(const rudder_weight* w, const uint16_t* X, int64_t ldx
         f.w_scales_t = w->scales_t; f.bias = bias; f.Y = Y; f.ldy = ldy;
         f.M = M; f.N = w->N; f.K = w->K; f.G = w->G;
         f.acc = acc; f.row0 = row0; f.rows = rows; f.col0 = col0; f.cols = cols;
-        if (launch_gemm_i8_fewrows(f, st) != cudaSuccess) return RUDDER_ERR_CUDA;
+        if ((gemm_i8_fewrows_applies(M, w->N, w->K, w->G) ? launch_gemm_i8_fewrows(f, st) : launch_gemm_i8_midrows(f, st)) != cudaSuccess) return RUDDER_ERR_CUDA;
         if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return RUDDER_ERR_CUDA;
         return RUDDER_OK;
     }
@@ -800,7 +800,7 @@ rudder_status rudder_quantize_activations(const rudder_weight* w, const uint16_t
     }
     // The kernel writes what production writes for this weight: int8, or (W4A4 on the E4M3 tensor path) the
     // E4M3 bytes of the same integers, which are then decoded in place so that the caller sees integers.
-    const bool e4m3 = w->f8 != 0 && !gemm_i8_fewrows_applies(M, w->N, w->K, w->G);     // the few-rows GEMM reads int8 whatever the weight layout
+    const bool e4m3 = w->f8 != 0 && !gemm_i8_register_path(M, w->N, w->K, w->G, w->f8 != 0);     // the register-level GEMMs read int8 whatever the weight layout
     if (launch_actq_int(a, qmax_of(w->scheme), e4m3, static_cast<int8_t*>(codes), w->K, row_scale, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     if (e4m3 && launch_e4m3_to_int8(static_cast<int8_t*>(codes), static_cast<size_t>(M) * w->K, static_cast<cudaStream_t>(stream)) != cudaSuccess)
@@ -825,7 +825,7 @@ rudder_status rudder_gelu_quantize_activations(const rudder_weight* w, const uin
     a.gamma_step = tab->gamma + static_cast<size_t>(step) * tab->S;
     a.clip_step = tab->clip + step;
     a.seg = sp;
-    const bool e4m3 = w->f8 != 0 && !gemm_i8_fewrows_applies(M, w->N, w->K, w->G);     // what production writes for this weight and shape
+    const bool e4m3 = w->f8 != 0 && !gemm_i8_register_path(M, w->N, w->K, w->G, w->f8 != 0);     // what production writes for this weight and shape
     if (launch_actq_gelu_static(a, qmax_of(w->scheme), e4m3, static_cast<int8_t*>(codes), w->K, row_scale, sm_count(), static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return RUDDER_ERR_CUDA;
     if (e4m3 && launch_e4m3_to_int8(static_cast<int8_t*>(codes), static_cast<size_t>(M) * w->K, static_cast<cudaStream_t>(stream)) != cudaSuccess)

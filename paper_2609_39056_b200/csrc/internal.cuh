@@ -158,5 +158,10 @@ struct GemmI8FewRowsArgs {
 };
 bool gemm_i8_fewrows_applies(int M, int N, int K, int G);
 cudaError_t launch_gemm_i8_fewrows(const GemmI8FewRowsArgs& a, cudaStream_t st);
+// A few dozen to a few hundred rows: register-level GEMM with shared-memory operand staging, see gemm_i8_midrows.cu.
+bool gemm_i8_midrows_applies(int M, int N, int K, int G, bool signmag);
+cudaError_t launch_gemm_i8_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st);
+// Either of the two: the prologue then writes int8 codes whatever the weight layout.
+inline bool gemm_i8_register_path(int M, int N, int K, int G, bool signmag) { return gemm_i8_fewrows_applies(M, N, K, G) || gemm_i8_midrows_applies(M, N, K, G, signmag); }
 
 }  // namespace rudder

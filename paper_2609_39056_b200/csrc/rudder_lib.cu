@@ -8,6 +8,7 @@
 #include "actq.cu"
 #include "gemm_i8.cu"
 #include "gemm_i8_fewrows.cu"
+#include "gemm_i8_midrows.cu"
 #include "gemm_fp4.cu"
 #include "gemm_fp4_pair.cu"
 #include "glue.cu"

@@ -111,6 +111,12 @@ CASES = [
     (200, 2304, 256, 128, "w4a4"),     # 64-token tiles, 18 stages
     (300, 640, 128, 64, "w4a4"),       # 256-token tiles with a ragged tail
     (64, 512, 256, 512, "w4a4"),       # G = K stays on the integer path
+    # the register-level kernel for a few dozen to a few hundred rows (groups of 64, K <= 2048), all three tile shapes
+    (512, 256, 1536, 64, "w4a8"),      # 128 x 64 tiles
+    (500, 384, 1536, 64, "w4a4"),      # the same with sign-magnitude weights and a ragged last token tile
+    (200, 640, 320, 64, "w4a8"),       # 64 x 32 tiles, ragged M
+    (70, 2048, 192, 64, "w4a4"),       # 16 stages: the copy ring wraps
+    (250, 1152, 2048, 64, "w4a8"),     # 64 x 64 tiles, 9 stages
 ]
 
 
