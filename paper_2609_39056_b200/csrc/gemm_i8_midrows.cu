@@ -88,19 +88,22 @@ __device__ __forceinline__ uint32_t mr_swz_a(uint32_t row) { return (row & 1u) |
 __device__ __forceinline__ uint32_t mr_swz_b(uint32_t row) { return row & 2u; }
 
 // WM = warps along the tokens (32 each), 8 / WM warps along the channels, NT = n8 tiles per warp:
-// the CTA owns BM = 32 WM tokens x BN = 8 NT (8 / WM) channels.
-template <int WM, int NT, bool SIGNMAG, bool DUMP, bool G64>
+// the CTA owns BM = 32 WM tokens x BN = 8 NT (8 / WM) channels.  Weight groups of 64 only: every 64-channel
+// block is a group.  (A second set of 8 warps per CTA that takes every other stage -- the loop is bound by
+// latency, and the small shapes have the registers -- measured 10 % slower: the barrier per stage grows.)
+template <int WM, int NT, bool SIGNMAG, bool DUMP>
 __global__ void __launch_bounds__(MR_THREADS, 1)
 gemm_i8_w4_midrows_kernel(const MidRowsParams p)
 {
+    constexpr int NTHR = MR_THREADS;
     constexpr int WNW = 8 / WM;
     constexpr int BM = 32 * WM;
     constexpr int BN = 8 * NT * WNW;
     constexpr int A_BYTES = BM * MR_KS;            // codes of one stage
     constexpr int B_BYTES = BN * MR_KS / 2;        // packed weights of one stage
-    constexpr int A_PIECES = BM * 8 / MR_THREADS;  // 16-byte pieces per thread and stage
+    constexpr int A_PIECES = BM * 8 / NTHR;        // 16-byte pieces per thread and stage
     constexpr int MR_NST = mr_stages(WM);
-    static_assert(BN * 4 <= MR_THREADS, "one weight piece per thread at most");
+    static_assert(BN * 4 <= NTHR && A_PIECES >= 1, "copy assignment");
     extern __shared__ __align__(128) uint8_t mr_smem[];
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -111,12 +114,11 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
     const int n0 = blockIdx.x * BN;
     const int m0 = blockIdx.y * BM;
     const int n_stages = p.K / MR_KS;
-    const int n_groups = p.K / p.G;
-    const int bpg = p.G >> 6;                      // 64-channel blocks per weight group
+    const int n_groups = p.K >> 6;
     const uint32_t smem0 = smem_u32(mr_smem);
     const uint32_t a_base = smem0;
     const uint32_t b_base = smem0 + MR_NST * A_BYTES;
-    float* scales_s = reinterpret_cast<float*>(mr_smem + MR_NST * (A_BYTES + B_BYTES));     // [K/G][BN]
+    float* scales_s = reinterpret_cast<float*>(mr_smem + MR_NST * (A_BYTES + B_BYTES));     // [K/64][BN]
     const float sc_mul = SIGNMAG ? 16.0f : 1.0f;   // sign-magnitude weights are the integers themselves, not 16 x
 
     // ---- what belongs to the weights: before waiting for the prologue kernel
@@ -128,7 +130,7 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
         if (b_thread) mr_cp16(b_base + (ks % MR_NST) * B_BYTES + b_dst, b_src + static_cast<size_t>(ks) * (MR_KS / 2));
     };
     for (int ks = 0; ks < MR_NST - 1 && ks < n_stages; ++ks) load_b(ks);
-    for (int i = tid; i < n_groups * BN; i += MR_THREADS) {
+    for (int i = tid; i < n_groups * BN; i += NTHR) {
         const int gg = i / BN, c = i - gg * BN;
         scales_s[i] = __ldg(p.scales_t + static_cast<size_t>(gg) * p.N + n0 + c) * sc_mul;
     }
@@ -136,7 +138,7 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
     uint32_t a_dst[A_PIECES];
 #pragma unroll
     for (int i = 0; i < A_PIECES; ++i) {
-        const int id = i * MR_THREADS + tid;
+        const int id = i * NTHR + tid;
         const int row = id >> 3, c = id & 7;
         const int tok = min(m0 + row, p.M - 1);    // rows past M repeat the last row (never stored)
         a_src[i] = p.codes + static_cast<size_t>(tok) * p.ldc + c * 16;
@@ -156,13 +158,13 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
     const uint32_t swa = mr_swz_a(g), swb = mr_swz_b(g);
     const uint32_t a_row0 = static_cast<uint32_t>(wm * 32 + g) * 128u + 8u * (q & 1);
     const uint32_t b_row0 = static_cast<uint32_t>(wn * 8 * NT + g) * 64u + 8u * (q & 1);
-    // G64: two sets of INT32 sums alternate between the two blocks of a stage, and a group is dequantised
-    // after the MMAs of the NEXT block have been issued: its own MMAs have long finished by then, so neither
-    // the conversions wait for the tensor pipe nor the next MMAs for the conversions.
+    // Two sets of INT32 sums alternate between the two blocks of a stage, and a group is dequantised after
+    // the MMAs of the NEXT block have been issued: its own MMAs have long finished by then, so neither the
+    // conversions wait for the tensor pipe nor the next MMAs for the conversions.
     // With fewer than four channel tiles per warp the two MMA steps of a block get accumulators of their own
     // (added at the group's end): otherwise the second step would wait out the first one's latency every time.
     constexpr int NS = (NT < 4) ? 2 : 1;
-    int C[G64 ? 2 : 1][NS][2][NT][4];
+    int C[2][NS][2][NT][4];
     float acc[2][NT][4];
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
@@ -172,7 +174,7 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
             for (int e = 0; e < 4; ++e) {
                 acc[mt][t][e] = 0.0f;
 #pragma unroll
-                for (int cs = 0; cs < (G64 ? 2 : 1); ++cs)
+                for (int cs = 0; cs < 2; ++cs)
 #pragma unroll
                     for (int st = 0; st < NS; ++st) C[cs][st][mt][t][e] = 0;
             }
@@ -202,8 +204,8 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
             }
         }
     };
-    // the MMAs of one 64-channel block of the stage at (a_st, b_st) into Cs; `fresh`: the block starts a group
-    auto block_mmas = [&](uint32_t a_st, uint32_t b_st, int blk, int (&Cs)[NS][2][NT][4], bool fresh) {
+    // the MMAs of one 64-channel block (= one weight group) of the stage at (a_st, b_st) into Cs, starting from zero
+    auto block_mmas = [&](uint32_t a_st, uint32_t b_st, int blk, int (&Cs)[NS][2][NT][4]) {
         const uint32_t ca = static_cast<uint32_t>(blk * 4 + 2 * (q >> 1));       // 16-byte piece of the low half of this lane's codes
         const uint32_t cb = static_cast<uint32_t>(blk * 2 + (q >> 1));
         uint2 a00[2], a01[2], a10[2], a11[2];
@@ -224,10 +226,7 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
             uint32_t b0, b1;
             mr_b_frag<SIGNMAG>(w[t].x, b0, b1);
 #pragma unroll
-            for (int mt = 0; mt < 2; ++mt) {
-                if (fresh) mr_mma_s8_first(Cs[0][mt][t], a00[mt].x, a10[mt].x, a01[mt].x, a11[mt].x, b0, b1);
-                else       mr_mma_s8(Cs[0][mt][t], a00[mt].x, a10[mt].x, a01[mt].x, a11[mt].x, b0, b1);
-            }
+            for (int mt = 0; mt < 2; ++mt) mr_mma_s8_first(Cs[0][mt][t], a00[mt].x, a10[mt].x, a01[mt].x, a11[mt].x, b0, b1);
         }
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
@@ -235,8 +234,8 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
             mr_b_frag<SIGNMAG>(w[t].y, b0, b1);
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
-                if (NS == 2 && fresh) mr_mma_s8_first(Cs[NS - 1][mt][t], a00[mt].y, a10[mt].y, a01[mt].y, a11[mt].y, b0, b1);
-                else                  mr_mma_s8(Cs[NS - 1][mt][t], a00[mt].y, a10[mt].y, a01[mt].y, a11[mt].y, b0, b1);
+                if (NS == 2) mr_mma_s8_first(Cs[NS - 1][mt][t], a00[mt].y, a10[mt].y, a01[mt].y, a11[mt].y, b0, b1);
+                else         mr_mma_s8(Cs[NS - 1][mt][t], a00[mt].y, a10[mt].y, a01[mt].y, a11[mt].y, b0, b1);
             }
         }
     };
@@ -248,23 +247,13 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
         mr_commit();
         const uint32_t a_st = a_base + (ks % MR_NST) * A_BYTES + a_row0;
         const uint32_t b_st = b_base + (ks % MR_NST) * B_BYTES + b_row0;
-        if (G64) {
-            block_mmas(a_st, b_st, 0, C[0], true);
-            if (ks > 0) dequant(C[G64 ? 1 : 0], 2 * ks - 1);
-            block_mmas(a_st, b_st, 1, C[G64 ? 1 : 0], true);
-            dequant(C[0], 2 * ks);
-        } else {
-            // groups of 128 and more end with a stage (an even number of blocks each)
-            const bool fresh = (2 * ks) % bpg == 0;
-            if (fresh) block_mmas(a_st, b_st, 0, C[0], true);
-            else       block_mmas(a_st, b_st, 0, C[0], false);
-            block_mmas(a_st, b_st, 1, C[0], false);
-            if ((2 * ks + 2) % bpg == 0) dequant(C[0], (2 * ks + 1) / bpg);
-        }
+        block_mmas(a_st, b_st, 0, C[0]);
+        if (ks > 0) dequant(C[1], 2 * ks - 1);
+        block_mmas(a_st, b_st, 1, C[1]);
+        dequant(C[0], 2 * ks);
     }
-    if (G64) dequant(C[G64 ? 1 : 0], 2 * n_stages - 1);
+    dequant(C[1], 2 * n_stages - 1);
     mr_wait<0>();
-
     // ---- row scale and bias (Eq. 10), bf16: a lane holds two adjacent channels of rows g and g + 8 per tile
     const bool pair_ok = ((p.ldy & 1) == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 3u) == 0);      // both channels in one 4-byte store
 #pragma unroll
@@ -312,10 +301,10 @@ static long long midrows_shape(int M, int N, int& wm, int& nt)
     }
     return best;
 }
-static size_t midrows_smem(int wm, int nt, int K, int G)
+static size_t midrows_smem(int wm, int nt, int K)
 {
     const int bm = 32 * wm, bn = 8 * nt * (8 / wm);
-    return static_cast<size_t>(mr_stages(wm)) * (bm * MR_KS + bn * MR_KS / 2) + static_cast<size_t>(K / G) * bn * sizeof(float);
+    return static_cast<size_t>(mr_stages(wm)) * (bm * MR_KS + bn * MR_KS / 2) + static_cast<size_t>(K / 64) * bn * sizeof(float);
 }
 
 // Where this kernel is the faster one (measured against the tcgen05 kernel with 64-token tiles and split K):
@@ -324,14 +313,14 @@ static size_t midrows_smem(int wm, int nt, int K, int G)
 // kernel wins again.
 bool gemm_i8_midrows_applies(int M, int N, int K, int G, bool signmag)
 {
-    if (!(M > 32 && M <= MR_MAX_M && K % MR_KS == 0 && N % 32 == 0 && G == 64 && K <= 2048)) return false;
+    if (!(M > 32 && M <= MR_MAX_M && K % MR_KS == 0 && N % 64 == 0 && G == 64 && K <= 2048)) return false;
     if (2.0 * M * N * K > (signmag ? 1.2e9 : 2.2e9)) return false;
     int wm, nt;
     const long long ctas = midrows_shape(M, N, wm, nt);
-    return ctas > 0 && ctas <= device_sm_count() && N % (8 * nt * (8 / wm)) == 0 && midrows_smem(wm, nt, K, G) <= 220 * 1024;
+    return ctas > 0 && ctas <= device_sm_count() && midrows_smem(wm, nt, K) <= 220 * 1024;
 }
 
-template <int WM, int NT, bool SIGNMAG, bool DUMP, bool G64>
+template <int WM, int NT, bool SIGNMAG, bool DUMP>
 static cudaError_t launch_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
 {
     MidRowsParams p;
@@ -339,8 +328,8 @@ static cudaError_t launch_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
     p.Y = a.Y; p.ldy = a.ldy; p.dump = a.acc; p.row0 = a.row0; p.rows = a.rows; p.col0 = a.col0; p.cols = a.cols;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.G;
     constexpr int BM = 32 * WM, BN = 8 * NT * (8 / WM);
-    const size_t smem = midrows_smem(WM, NT, a.K, a.G);
-    cudaError_t e = cudaFuncSetAttribute(gemm_i8_w4_midrows_kernel<WM, NT, SIGNMAG, DUMP, G64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    const size_t smem = midrows_smem(WM, NT, a.K);
+    cudaError_t e = cudaFuncSetAttribute(gemm_i8_w4_midrows_kernel<WM, NT, SIGNMAG, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.N / BN, (a.M + BM - 1) / BM, 1);
@@ -352,7 +341,7 @@ static cudaError_t launch_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_midrows_kernel<WM, NT, SIGNMAG, DUMP, G64>, p);
+    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_midrows_kernel<WM, NT, SIGNMAG, DUMP>, p);
 }
 
 cudaError_t launch_gemm_i8_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
@@ -360,14 +349,12 @@ cudaError_t launch_gemm_i8_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
     const bool dump = a.acc != nullptr;
     int wm, nt;
     midrows_shape(a.M, a.N, wm, nt);
-#define RUDDER_MR_LAUNCH2(WM, NT, G64)                                                                                              \
-    return a.signmag ? (dump ? launch_midrows<WM, NT, true, true, G64>(a, st) : launch_midrows<WM, NT, true, false, G64>(a, st))    \
-                     : (dump ? launch_midrows<WM, NT, false, true, G64>(a, st) : launch_midrows<WM, NT, false, false, G64>(a, st));
-#define RUDDER_MR_LAUNCH(WM, NT) if (a.G == 64) { RUDDER_MR_LAUNCH2(WM, NT, true) } else { RUDDER_MR_LAUNCH2(WM, NT, false) }
+#define RUDDER_MR_LAUNCH(WM, NT)                                                                                          \
+    return a.signmag ? (dump ? launch_midrows<WM, NT, true, true>(a, st) : launch_midrows<WM, NT, true, false>(a, st))    \
+                     : (dump ? launch_midrows<WM, NT, false, true>(a, st) : launch_midrows<WM, NT, false, false>(a, st));
     if (wm == 4) { RUDDER_MR_LAUNCH(4, 4) }
     if (nt == 2) { RUDDER_MR_LAUNCH(2, 2) }
     RUDDER_MR_LAUNCH(2, 1)
-#undef RUDDER_MR_LAUNCH2
 #undef RUDDER_MR_LAUNCH
 }
 
