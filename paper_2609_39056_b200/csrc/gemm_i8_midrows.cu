@@ -10,7 +10,7 @@
 //   * a CTA of 8 warps owns BM tokens x BN output channels over all of K; a warp owns 32 tokens x 8 NT
 //     channels (two m16 tiles x NT n8 tiles of mma.sync.m16n8k32.s8);
 //   * codes Q_X (int8, from the prologue kernel) and packed 4-bit weights are staged through a ring of
-//     shared-memory stages of 128 input channels by 16-byte cp.async copies; the weight copies of the
+//     shared-memory stages of 256 input channels by 16-byte cp.async copies; the weight copies of the
 //     first stages and the group scales of the CTA's channels are requested BEFORE waiting for the
 //     prologue kernel (programmatic dependent launch);
 //   * fragments are 8-byte shared-memory loads in the layout the few-rows kernel uses (the packed weight
@@ -28,10 +28,11 @@ namespace rudder {
 namespace {
 
 constexpr int MR_THREADS = 256;
-constexpr int MR_KS = 128;             // input channels per stage
+constexpr int MR_KS = 256;             // input channels per stage (128 measured 5-9 % slower: twice the barriers)
 // Stages in the ring: what is in flight per SM has to cover an L2 round trip per stage, so as many as fit.
-__host__ __device__ constexpr int mr_stages(int wm) { return wm == 4 ? 8 : 12; }
+__host__ __device__ constexpr int mr_stages(int wm) { return wm == 4 ? 4 : 6; }
 constexpr int MR_MAX_M = 512;          // rows up to which this kernel is considered
+constexpr int MR_MAX_K = 4096;         // and row length
 
 struct MidRowsParams {
     const int8_t* codes; int64_t ldc;  // Q_X int8 [M, ldc]
@@ -85,7 +86,7 @@ __device__ __forceinline__ void mr_b_frag(uint32_t pk, uint32_t& b0, uint32_t& b
 }
 // Permutation of the 16-byte pieces of a code row (8 pieces per stage) / weight row (4 pieces per stage).
 __device__ __forceinline__ uint32_t mr_swz_a(uint32_t row) { return (row & 1u) | ((row & 2u) << 1); }
-__device__ __forceinline__ uint32_t mr_swz_b(uint32_t row) { return row & 2u; }
+__device__ __forceinline__ uint32_t mr_swz_b(uint32_t row) { return (row & 3u) << 1; }
 
 // WM = warps along the tokens (32 each), 8 / WM warps along the channels, NT = n8 tiles per warp:
 // the CTA owns BM = 32 WM tokens x BN = 8 NT (8 / WM) channels.  Weight groups of 64 only: every 64-channel
@@ -101,9 +102,11 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
     constexpr int BN = 8 * NT * WNW;
     constexpr int A_BYTES = BM * MR_KS;            // codes of one stage
     constexpr int B_BYTES = BN * MR_KS / 2;        // packed weights of one stage
-    constexpr int A_PIECES = BM * 8 / NTHR;        // 16-byte pieces per thread and stage
+    constexpr int A_PIECES = BM * (MR_KS / 16) / NTHR;        // 16-byte pieces per thread and stage
+    constexpr int B_ALL = BN * (MR_KS / 32);       // 16-byte weight pieces per stage
+    constexpr int B_PIECES = (B_ALL + NTHR - 1) / NTHR;
     constexpr int MR_NST = mr_stages(WM);
-    static_assert(BN * 4 <= NTHR && A_PIECES >= 1, "copy assignment");
+    static_assert(A_PIECES >= 1, "copy assignment");
     extern __shared__ __align__(128) uint8_t mr_smem[];
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -122,12 +125,22 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
     const float sc_mul = SIGNMAG ? 16.0f : 1.0f;   // sign-magnitude weights are the integers themselves, not 16 x
 
     // ---- what belongs to the weights: before waiting for the prologue kernel
-    const bool b_thread = tid < BN * 4;
-    const int b_row = tid >> 2, b_c = tid & 3;
-    const uint8_t* b_src = p.wq + static_cast<size_t>(n0 + (b_thread ? b_row : 0)) * (p.K >> 1) + b_c * 16;
-    const uint32_t b_dst = static_cast<uint32_t>(b_row) * 64u + ((static_cast<uint32_t>(b_c) ^ mr_swz_b(b_row)) << 4);
+    constexpr int BPR = MR_KS / 32;                // weight pieces per channel row
+    const uint8_t* b_src[B_PIECES];
+    uint32_t b_dst[B_PIECES];
+    bool b_on[B_PIECES];
+#pragma unroll
+    for (int i = 0; i < B_PIECES; ++i) {
+        const int id = i * NTHR + tid;
+        b_on[i] = id < B_ALL;
+        const int row = b_on[i] ? id / BPR : 0, c = id % BPR;
+        b_src[i] = p.wq + static_cast<size_t>(n0 + row) * (p.K >> 1) + c * 16;
+        b_dst[i] = static_cast<uint32_t>(row) * (MR_KS / 2) + ((static_cast<uint32_t>(c) ^ mr_swz_b(row)) << 4);
+    }
     auto load_b = [&](int ks) {
-        if (b_thread) mr_cp16(b_base + (ks % MR_NST) * B_BYTES + b_dst, b_src + static_cast<size_t>(ks) * (MR_KS / 2));
+#pragma unroll
+        for (int i = 0; i < B_PIECES; ++i)
+            if (b_on[i]) mr_cp16(b_base + (ks % MR_NST) * B_BYTES + b_dst[i], b_src[i] + static_cast<size_t>(ks) * (MR_KS / 2));
     };
     for (int ks = 0; ks < MR_NST - 1 && ks < n_stages; ++ks) load_b(ks);
     for (int i = tid; i < n_groups * BN; i += NTHR) {
@@ -139,10 +152,10 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
 #pragma unroll
     for (int i = 0; i < A_PIECES; ++i) {
         const int id = i * NTHR + tid;
-        const int row = id >> 3, c = id & 7;
+        const int row = id / (MR_KS / 16), c = id % (MR_KS / 16);
         const int tok = min(m0 + row, p.M - 1);    // rows past M repeat the last row (never stored)
         a_src[i] = p.codes + static_cast<size_t>(tok) * p.ldc + c * 16;
-        a_dst[i] = static_cast<uint32_t>(row) * 128u + ((static_cast<uint32_t>(c) ^ mr_swz_a(row)) << 4);
+        a_dst[i] = static_cast<uint32_t>(row) * MR_KS + ((static_cast<uint32_t>(c) ^ mr_swz_a(row)) << 4);
     }
     auto load_a = [&](int ks) {
 #pragma unroll
@@ -156,8 +169,8 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
 
     // fragment addresses inside a stage (without the 64-channel block's piece offset, which is XORed in below)
     const uint32_t swa = mr_swz_a(g), swb = mr_swz_b(g);
-    const uint32_t a_row0 = static_cast<uint32_t>(wm * 32 + g) * 128u + 8u * (q & 1);
-    const uint32_t b_row0 = static_cast<uint32_t>(wn * 8 * NT + g) * 64u + 8u * (q & 1);
+    const uint32_t a_row0 = static_cast<uint32_t>(wm * 32 + g) * MR_KS + 8u * (q & 1);
+    const uint32_t b_row0 = static_cast<uint32_t>(wn * 8 * NT + g) * (MR_KS / 2) + 8u * (q & 1);
     // Two sets of INT32 sums alternate between the two blocks of a stage, and a group is dequantised after
     // the MMAs of the NEXT block have been issued: its own MMAs have long finished by then, so neither the
     // conversions wait for the tensor pipe nor the next MMAs for the conversions.
@@ -211,15 +224,15 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
         uint2 a00[2], a01[2], a10[2], a11[2];
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
-            const uint32_t r = a_st + mt * 16 * 128;
+            const uint32_t r = a_st + mt * 16 * MR_KS;
             a00[mt] = mr_lds8(r + ((ca ^ swa) << 4));
             a01[mt] = mr_lds8(r + (((ca + 1) ^ swa) << 4));
-            a10[mt] = mr_lds8(r + 8 * 128 + ((ca ^ swa) << 4));
-            a11[mt] = mr_lds8(r + 8 * 128 + (((ca + 1) ^ swa) << 4));
+            a10[mt] = mr_lds8(r + 8 * MR_KS + ((ca ^ swa) << 4));
+            a11[mt] = mr_lds8(r + 8 * MR_KS + (((ca + 1) ^ swa) << 4));
         }
         uint2 w[NT];
 #pragma unroll
-        for (int t = 0; t < NT; ++t) w[t] = mr_lds8(b_st + t * 8 * 64 + ((cb ^ swb) << 4));
+        for (int t = 0; t < NT; ++t) w[t] = mr_lds8(b_st + t * 8 * (MR_KS / 2) + ((cb ^ swb) << 4));
         // first MMA step of every tile, then the second: consecutive MMAs never share an accumulator
 #pragma unroll
         for (int t = 0; t < NT; ++t) {
@@ -247,12 +260,14 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
         mr_commit();
         const uint32_t a_st = a_base + (ks % MR_NST) * A_BYTES + a_row0;
         const uint32_t b_st = b_base + (ks % MR_NST) * B_BYTES + b_row0;
-        block_mmas(a_st, b_st, 0, C[0]);
-        if (ks > 0) dequant(C[1], 2 * ks - 1);
-        block_mmas(a_st, b_st, 1, C[1]);
-        dequant(C[0], 2 * ks);
+        constexpr int BPS = MR_KS / 64;                      // blocks (= weight groups) per stage
+#pragma unroll
+        for (int blk = 0; blk < BPS; ++blk) {
+            block_mmas(a_st, b_st, blk, C[blk & 1]);
+            if (ks > 0 || blk > 0) dequant(C[(blk & 1) ^ 1], ks * BPS + blk - 1);
+        }
     }
-    dequant(C[1], 2 * n_stages - 1);
+    dequant(C[1], n_groups - 1);
     mr_wait<0>();
     // ---- row scale and bias (Eq. 10), bf16: a lane holds two adjacent channels of rows g and g + 8 per tile
     const bool pair_ok = ((p.ldy & 1) == 0) && ((reinterpret_cast<uintptr_t>(p.Y) & 3u) == 0);      // both channels in one 4-byte store
@@ -308,12 +323,12 @@ static size_t midrows_smem(int wm, int nt, int K)
 }
 
 // Where this kernel is the faster one (measured against the tcgen05 kernel with 64-token tiles and split K):
-// weight groups of 64, rows of up to 2048 channels, one wave of CTAs, and little work in all -- its MMAs run at
-// the legacy rate, so beyond about 2 GOP (1.2 with the costlier sign-magnitude fragments) the tensor-memory
-// kernel wins again.
+// weight groups of 64, rows of up to 4096 channels (8192: slower), one wave of CTAs, and little work in all --
+// its MMAs run at the legacy rate, so beyond about 2 GOP (1.2 with the costlier sign-magnitude fragments) the
+// tensor-memory kernel wins again (level at 4 GOP).
 bool gemm_i8_midrows_applies(int M, int N, int K, int G, bool signmag)
 {
-    if (!(M > 32 && M <= MR_MAX_M && K % MR_KS == 0 && N % 64 == 0 && G == 64 && K <= 2048)) return false;
+    if (!(M > 32 && M <= MR_MAX_M && K % MR_KS == 0 && N % 64 == 0 && G == 64 && K <= MR_MAX_K)) return false;
     if (2.0 * M * N * K > (signmag ? 1.2e9 : 2.2e9)) return false;
     int wm, nt;
     const long long ctas = midrows_shape(M, N, wm, nt);

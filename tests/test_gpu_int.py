@@ -115,8 +115,8 @@ CASES = [
     (512, 256, 1536, 64, "w4a8"),      # 128 x 64 tiles
     (500, 384, 1536, 64, "w4a4"),      # the same with sign-magnitude weights and a ragged last token tile
     (200, 640, 320, 64, "w4a8"),       # 64 x 32 tiles, ragged M
-    (70, 2048, 192, 64, "w4a4"),       # 16 stages: the copy ring wraps
-    (250, 1152, 2048, 64, "w4a8"),     # 64 x 64 tiles, 9 stages
+    (70, 2048, 192, 64, "w4a4"),       # 8 stages: the copy ring wraps
+    (250, 1280, 2048, 64, "w4a8"),     # 64 x 64 tiles, 5 stages
 ]
 
 
