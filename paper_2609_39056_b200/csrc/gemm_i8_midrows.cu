@@ -27,7 +27,6 @@ namespace rudder {
 
 namespace {
 
-constexpr int MR_THREADS = 256;
 constexpr int MR_KS = 256;             // input channels per stage (128 measured 5-9 % slower: twice the barriers)
 // Stages in the ring: what is in flight per SM has to cover an L2 round trip per stage, so as many as fit.
 __host__ __device__ constexpr int mr_stages(int wm) { return wm == 4 ? 4 : 6; }
@@ -92,12 +91,12 @@ __device__ __forceinline__ uint32_t mr_swz_b(uint32_t row) { return (row & 3u) <
 // the CTA owns BM = 32 WM tokens x BN = 8 NT (8 / WM) channels.  Weight groups of 64 only: every 64-channel
 // block is a group.  (A second set of 8 warps per CTA that takes every other stage -- the loop is bound by
 // latency, and the small shapes have the registers -- measured 10 % slower: the barrier per stage grows.)
-template <int WM, int NT, bool SIGNMAG, bool DUMP>
-__global__ void __launch_bounds__(MR_THREADS, 1)
+template <int WM, int NT, int NW, bool SIGNMAG, bool DUMP>
+__global__ void __launch_bounds__(32 * NW, 1)
 gemm_i8_w4_midrows_kernel(const MidRowsParams p)
 {
-    constexpr int NTHR = MR_THREADS;
-    constexpr int WNW = 8 / WM;
+    constexpr int NTHR = 32 * NW;
+    constexpr int WNW = NW / WM;
     constexpr int BM = 32 * WM;
     constexpr int BN = 8 * NT * WNW;
     constexpr int A_BYTES = BM * MR_KS;            // codes of one stage
@@ -298,27 +297,29 @@ gemm_i8_w4_midrows_kernel(const MidRowsParams p)
 
 }  // namespace
 
-// Tile shapes, largest first: {warps along the tokens, n8 tiles per warp} -> BM = 32 WM, BN = 8 NT (8 / WM).
-// The largest shape that still gives at least 0.6 CTAs per SM; failing that the one with the most CTAs.
-// Returns the number of CTAs.
-static long long midrows_shape(int M, int N, int& wm, int& nt)
+// Tile shapes, largest first: {warps along the tokens, n8 tiles per warp, warps} -> BM = 32 WM,
+// BN = 8 NT (warps / WM).  The largest shape that still gives at least 0.6 CTAs per SM; failing that the one
+// with the most CTAs (the last one, 64 x 16 with four warps, is there for the smallest layers).  Returns the
+// number of CTAs.
+constexpr int kMidShapes[4][3] = {{4, 4, 8}, {2, 2, 8}, {2, 1, 8}, {2, 1, 4}};
+static long long midrows_shape(int M, int N, int& idx)
 {
     const int sms = device_sm_count();
-    const int cand[3][2] = {{4, 4}, {2, 2}, {2, 1}};
     long long best = -1;
-    wm = 2; nt = 1;
-    for (int i = 0; i < 3; ++i) {
-        const int bm = 32 * cand[i][0], bn = 8 * cand[i][1] * (8 / cand[i][0]);
+    idx = 3;
+    for (int i = 0; i < 4; ++i) {
+        const int bm = 32 * kMidShapes[i][0], bn = 8 * kMidShapes[i][1] * (kMidShapes[i][2] / kMidShapes[i][0]);
         if (N % bn != 0 || (i == 0 && M <= 64)) continue;
         const long long ctas = static_cast<long long>((M + bm - 1) / bm) * (N / bn);
-        if (ctas * 10 >= 6LL * sms) { wm = cand[i][0]; nt = cand[i][1]; return ctas; }
-        if (ctas > best) { best = ctas; wm = cand[i][0]; nt = cand[i][1]; }
+        if (ctas > sms) continue;
+        if (ctas * 10 >= 6LL * sms) { idx = i; return ctas; }
+        if (ctas > best) { best = ctas; idx = i; }
     }
     return best;
 }
-static size_t midrows_smem(int wm, int nt, int K)
+static size_t midrows_smem(int wm, int nt, int nw, int K)
 {
-    const int bm = 32 * wm, bn = 8 * nt * (8 / wm);
+    const int bm = 32 * wm, bn = 8 * nt * (nw / wm);
     return static_cast<size_t>(mr_stages(wm)) * (bm * MR_KS + bn * MR_KS / 2) + static_cast<size_t>(K / 64) * bn * sizeof(float);
 }
 
@@ -330,25 +331,25 @@ bool gemm_i8_midrows_applies(int M, int N, int K, int G, bool signmag)
 {
     if (!(M > 32 && M <= MR_MAX_M && K % MR_KS == 0 && N % 64 == 0 && G == 64 && K <= MR_MAX_K)) return false;
     if (2.0 * M * N * K > (signmag ? 1.2e9 : 2.2e9)) return false;
-    int wm, nt;
-    const long long ctas = midrows_shape(M, N, wm, nt);
-    return ctas > 0 && ctas <= device_sm_count() && midrows_smem(wm, nt, K) <= 220 * 1024;
+    int idx;
+    const long long ctas = midrows_shape(M, N, idx);
+    return ctas > 0 && midrows_smem(kMidShapes[idx][0], kMidShapes[idx][1], kMidShapes[idx][2], K) <= 220 * 1024;
 }
 
-template <int WM, int NT, bool SIGNMAG, bool DUMP>
+template <int WM, int NT, int NW, bool SIGNMAG, bool DUMP>
 static cudaError_t launch_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
 {
     MidRowsParams p;
     p.codes = a.codes; p.ldc = a.ldc; p.row_scale = a.row_scale; p.wq = a.wq; p.scales_t = a.w_scales_t; p.bias = a.bias;
     p.Y = a.Y; p.ldy = a.ldy; p.dump = a.acc; p.row0 = a.row0; p.rows = a.rows; p.col0 = a.col0; p.cols = a.cols;
     p.M = a.M; p.N = a.N; p.K = a.K; p.G = a.G;
-    constexpr int BM = 32 * WM, BN = 8 * NT * (8 / WM);
-    const size_t smem = midrows_smem(WM, NT, a.K);
-    cudaError_t e = cudaFuncSetAttribute(gemm_i8_w4_midrows_kernel<WM, NT, SIGNMAG, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    constexpr int BM = 32 * WM, BN = 8 * NT * (NW / WM);
+    const size_t smem = midrows_smem(WM, NT, NW, a.K);
+    cudaError_t e = cudaFuncSetAttribute(gemm_i8_w4_midrows_kernel<WM, NT, NW, SIGNMAG, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.N / BN, (a.M + BM - 1) / BM, 1);
-    cfg.blockDim = dim3(MR_THREADS, 1, 1);
+    cfg.blockDim = dim3(32 * NW, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -356,20 +357,21 @@ static cudaError_t launch_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_midrows_kernel<WM, NT, SIGNMAG, DUMP>, p);
+    return cudaLaunchKernelEx(&cfg, gemm_i8_w4_midrows_kernel<WM, NT, NW, SIGNMAG, DUMP>, p);
 }
 
 cudaError_t launch_gemm_i8_midrows(const GemmI8FewRowsArgs& a, cudaStream_t st)
 {
     const bool dump = a.acc != nullptr;
-    int wm, nt;
-    midrows_shape(a.M, a.N, wm, nt);
-#define RUDDER_MR_LAUNCH(WM, NT)                                                                                          \
-    return a.signmag ? (dump ? launch_midrows<WM, NT, true, true>(a, st) : launch_midrows<WM, NT, true, false>(a, st))    \
-                     : (dump ? launch_midrows<WM, NT, false, true>(a, st) : launch_midrows<WM, NT, false, false>(a, st));
-    if (wm == 4) { RUDDER_MR_LAUNCH(4, 4) }
-    if (nt == 2) { RUDDER_MR_LAUNCH(2, 2) }
-    RUDDER_MR_LAUNCH(2, 1)
+    int idx;
+    midrows_shape(a.M, a.N, idx);
+#define RUDDER_MR_LAUNCH(WM, NT, NW)                                                                                              \
+    return a.signmag ? (dump ? launch_midrows<WM, NT, NW, true, true>(a, st) : launch_midrows<WM, NT, NW, true, false>(a, st))    \
+                     : (dump ? launch_midrows<WM, NT, NW, false, true>(a, st) : launch_midrows<WM, NT, NW, false, false>(a, st));
+    if (idx == 0) { RUDDER_MR_LAUNCH(4, 4, 8) }
+    if (idx == 1) { RUDDER_MR_LAUNCH(2, 2, 8) }
+    if (idx == 2) { RUDDER_MR_LAUNCH(2, 1, 8) }
+    RUDDER_MR_LAUNCH(2, 1, 4)
 #undef RUDDER_MR_LAUNCH
 }
 

@@ -111,12 +111,14 @@ CASES = [
     (200, 2304, 256, 128, "w4a4"),     # 64-token tiles, 18 stages
     (300, 640, 128, 64, "w4a4"),       # 256-token tiles with a ragged tail
     (64, 512, 256, 512, "w4a4"),       # G = K stays on the integer path
-    # the register-level kernel for a few dozen to a few hundred rows (groups of 64, K <= 2048), all three tile shapes
+    # the register-level kernel for a few dozen to a few hundred rows (groups of 64, K a multiple of 256 up to 4096),
+    # all four tile shapes
     (512, 256, 1536, 64, "w4a8"),      # 128 x 64 tiles
-    (500, 384, 1536, 64, "w4a4"),      # the same with sign-magnitude weights and a ragged last token tile
-    (200, 640, 320, 64, "w4a8"),       # 64 x 32 tiles, ragged M
-    (70, 2048, 192, 64, "w4a4"),       # 8 stages: the copy ring wraps
+    (500, 512, 1536, 64, "w4a4"),      # the same with sign-magnitude weights and a ragged last token tile
     (250, 1280, 2048, 64, "w4a8"),     # 64 x 64 tiles, 5 stages
+    (60, 512, 3072, 64, "w4a8"),       # 64 x 32 tiles
+    (200, 768, 320, 64, "w4a8"),       # 64 x 16 tiles with four warps, ragged M
+    (70, 2048, 192, 64, "w4a4"),       # the same, 8 stages: the copy ring wraps
 ]
 
 
