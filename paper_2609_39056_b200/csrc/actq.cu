@@ -565,7 +565,7 @@ __global__ void __launch_bounds__(NCH == 1 ? 1024 : (NCH == 2 ? 512 : 256)) actq
             continue;
         }
         const int slot = j & (kRowSlots - 1);
-        // A thread whose wait gave up still walks to the row's barrier, where the verdict becomes common to
+        // A thread whose wait gave up still walks to the row's barrier, where the outcome becomes common to
         // the CTA (what it computes from the unfinished row meanwhile is discarded).
         bool ok = mbar_wait<20>(bar0 + 8u * slot, (j / kRowSlots) & 1, &abort_word, W_ROW_FULL);
         const float g = g_slot[slot];

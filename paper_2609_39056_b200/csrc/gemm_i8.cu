@@ -549,7 +549,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
             const float sc = n_ok ? sc_next * sc_mul : 0.0f;
             sc_next = sc_next2;
             if (g + 2 < n_groups) sc_next2 = ldg_f32_volatile(sc_ptr + static_cast<size_t>(g + 2) * p.N);
-            // the verdict is made warp-uniform (the TMEM loads below are warp-collective)
+            // the outcome is made warp-uniform (the TMEM loads below are warp-collective)
             // every lane polls: a single polling lane followed by a shuffle measured 10 % slower per group
             ok = mbar_wait<RUDDER_SLEEP_EPI>(acc_full(buf), phb, abortp, W_ACC_FULL);
             ok = __all_sync(0xffffffffu, ok);
@@ -610,7 +610,7 @@ gemm_i8_w4_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constan
 #pragma unroll
             for (int pass = 0; pass < 2; ++pass) {
                 if (threadIdx.x == 256) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                // the barrier also makes the verdict common to all drain threads: they leave the tile loop together
+                // the barrier also makes the outcome common to all drain threads: they leave the tile loop together
                 ok = bar_sync_and(1, EPI_THREADS, ok);
                 if (ok) {
                     if (ch_local < p.out_pitch) {

@@ -71,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 
 // Named barrier over `count` threads that also ANDs a predicate across them: every participant gets the
-// same verdict, so a role that gave up a bounded wait takes the whole group out of its loop together
+// same outcome, so a role that gave up a bounded wait takes the whole group out of its loop together
 // (a thread that left alone would strand the others at their next barrier).
 __device__ __forceinline__ bool bar_sync_and(int id, int count, bool pred) {
     uint32_t r;

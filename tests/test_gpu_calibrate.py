@@ -1,6 +1,6 @@
 """The GPU-side toy calibrator (Eq. 9) against the oracle's: the objective it evaluates through
 `rudder_linear` agrees with the oracle's at fixed points, and the point it finds is as good as the
-oracle's own when both are judged by the oracle's objective."""
+oracle's own when both are scored by the oracle's objective."""
 import numpy as np
 import pytest
 import torch
