@@ -7,8 +7,8 @@
 // math), while wider tiles move the bound to the per-group drain of tensor memory.  Here the per-group
 // INT32 sums stay in registers, as Eq. 10 with group scales wants them:
 //
-//   * a CTA of 8 warps owns BM tokens x BN output channels over all of K; a warp owns 32 tokens x 8 NT
-//     channels (two m16 tiles x NT n8 tiles of mma.sync.m16n8k32.s8);
+//   * a CTA of 8 (or 4) warps owns BM tokens x BN output channels over all of K; a warp owns 32 tokens x
+//     8 NT channels (two m16 tiles x NT n8 tiles of mma.sync.m16n8k32.s8);
 //   * codes Q_X (int8, from the prologue kernel) and packed 4-bit weights are staged through a ring of
 //     shared-memory stages of 256 input channels by 16-byte cp.async copies; the weight copies of the
 //     first stages and the group scales of the CTA's channels are requested BEFORE waiting for the
@@ -17,8 +17,10 @@
 //     word is the B fragment: one shift and two masks; sign-magnitude layout: two byte permutes and a
 //     per-byte negate); both tiles are stored with their 16-byte pieces permuted by row so that the loads
 //     of a half warp fall into 16 different bank pairs;
-//   * at the end of each weight group: fp32(C) * Delta_W[j,g] added into fp32 registers, C cleared; at the
-//     end of K: * r_i + b_j, bf16.  No tensor memory, no split K, no scratch.
+//   * at the end of each weight group (64 channels): fp32(C) * Delta_W[j,g] added into fp32 registers; the
+//     next group starts from a zero accumulator in a second set of registers, so that the conversions of one
+//     group run under the MMAs of the next; at the end of K: * r_i + b_j, bf16.  No tensor memory, no split K,
+//     no scratch.
 #include "internal.cuh"
 
 #include <cuda_bf16.h>
@@ -83,12 +85,14 @@ __device__ __forceinline__ void mr_b_frag(uint32_t pk, uint32_t& b0, uint32_t& b
         b1 = pk & 0xF0F0F0F0u;
     }
 }
-// Permutation of the 16-byte pieces of a code row (8 pieces per stage) / weight row (4 pieces per stage).
+// Permutation of the 16-byte pieces of a code row (16 pieces per stage; bits 0 and 2 of the piece index) and of
+// a weight row (8 pieces per stage), each a function of the row so that the fragment loads of a half warp (four
+// rows x four lanes, 8 bytes each) cover 16 different bank pairs.
 __device__ __forceinline__ uint32_t mr_swz_a(uint32_t row) { return (row & 1u) | ((row & 2u) << 1); }
 __device__ __forceinline__ uint32_t mr_swz_b(uint32_t row) { return (row & 3u) << 1; }
 
-// WM = warps along the tokens (32 each), 8 / WM warps along the channels, NT = n8 tiles per warp:
-// the CTA owns BM = 32 WM tokens x BN = 8 NT (8 / WM) channels.  Weight groups of 64 only: every 64-channel
+// WM = warps along the tokens (32 each), NW / WM warps along the channels, NT = n8 tiles per warp:
+// the CTA owns BM = 32 WM tokens x BN = 8 NT (NW / WM) channels.  Weight groups of 64 only: every 64-channel
 // block is a group.  (A second set of 8 warps per CTA that takes every other stage -- the loop is bound by
 // latency, and the small shapes have the registers -- measured 10 % slower: the barrier per stage grows.)
 template <int WM, int NT, int NW, bool SIGNMAG, bool DUMP>
